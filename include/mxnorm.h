@@ -1,0 +1,143 @@
+/*
+ * libmxnorm - C ABI of the B200 (sm_100a) MXNorm hot path.
+ *
+ * MXNorm (Algorithm 2 of the paper) replaces "RMSNorm followed by an MXFP8 cast"
+ * (Algorithm 1) by one pass that takes every block's absmax, estimates the row RMS
+ * from those K = D/B block statistics and emits the normalised tensor directly as
+ * block-scaled low-precision codes.
+ *
+ * Conventions shared by every entry point unless stated otherwise
+ * ----------------------------------------------------------------
+ *  - Tensor pointers are DEVICE pointers owned by the caller.  The library never
+ *    allocates, frees or synchronises; work is enqueued on `cuda_stream` (a
+ *    cudaStream_t passed as void*, NULL = the legacy default stream) of the
+ *    device that is current when the call is made.
+ *  - X is bf16 [T, D], row-major, contiguous, base address 16-byte aligned.
+ *    T >= 0 rows (tokens), D hidden size, `block` = B, K = D / B blocks per row.
+ *    Supported: B in {16, 32, 64} (NVFP4: B = 16 fixed), D % B == 0,
+ *    D <= 32768 * B / 32.  T == 0 returns MXN_OK without a launch.
+ *  - codes: one byte per element (E4M3, OCP "fn": bias 7, max 448, no infinity),
+ *    [T, D] row-major; written with 32-byte stores: base 32-byte aligned.
+ *  - scales: one byte per block.  MXN_SCALES_ROWMAJOR: [T, K].
+ *    MXN_SCALES_SWIZZLE_128x4: the tiled layout block-scaled tensor-core GEMMs
+ *    read - rows padded to a multiple of 128, scale columns to a multiple of 4,
+ *    each (128 rows x 4 scales) tile 512 contiguous bytes, tiles row-tile major;
+ *    byte offset of (r, c) =
+ *      ((r/128) * ceil(K/4) + c/4) * 512 + (r%32) * 16 + ((r%128)/32) * 4 + c%4.
+ *    The buffer must hold mxn_scale_bytes(T, K, layout) bytes; padding bytes are
+ *    written as 0.
+ *  - Outputs are fully overwritten.  Inputs must be finite; results for NaN/Inf
+ *    inputs are unspecified (no fault).
+ *  - Every function returns a status; nothing aborts, throws or prints.  Argument
+ *    errors are detected before anything is enqueued.  CUDA launch failures map
+ *    to MXN_ERR_CUDA.
+ *  - Arithmetic contract (what the CPU oracle states and the tests compare):
+ *    block absmaxes exact; row statistic accumulated in binary64 and rounded once
+ *    to binary32; every element-wise product one IEEE binary32 operation; E8M0
+ *    scales by exact exponent tests; element codes round-to-nearest-even,
+ *    saturating.
+ */
+#ifndef MXNORM_H_
+#define MXNORM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MXN_OK = 0,
+    MXN_ERR_NULL = 1,      /* a required pointer is NULL */
+    MXN_ERR_SHAPE = 2,     /* T < 0, D <= 0, D % B != 0, unsupported B or D, bad p */
+    MXN_ERR_ALIGN = 3,     /* a pointer misses the alignment stated above */
+    MXN_ERR_ENUM = 4,      /* unknown rounding mode / layout */
+    MXN_ERR_WORKSPACE = 5, /* workspace NULL or smaller than the query says */
+    MXN_ERR_CUDA = 6,      /* the CUDA runtime reported an error at launch */
+    MXN_ERR_TIMEOUT = 7    /* reserved: a bounded device-side wait ran out */
+} mxn_status;
+
+/* Power-of-two rounding of the block scale (Section 3.2: "implementation-defined").
+ *   RCEIL_POW2 : the paper's rule - round UP the quotient absmax / 2^emax, where 2^emax
+ *                is the largest power of two of the element format (256 for E4M3):
+ *                S = 2^(ceil(log2 absmax) - emax).  Codes never exceed 2^emax.
+ *   FLOOR_OCP  : S = 2^(floor(log2 absmax) - emax) (OCP MX specification); codes saturate.
+ *   RCEIL_MAX  : S = 2^ceil(log2(absmax / max_elem)) with max_elem = 448 (one binary32
+ *                division). */
+typedef enum { MXN_ROUND_RCEIL_POW2 = 0, MXN_ROUND_FLOOR_OCP = 1, MXN_ROUND_RCEIL_MAX = 2 } mxn_round;
+
+typedef enum { MXN_SCALES_ROWMAJOR = 0, MXN_SCALES_SWIZZLE_128x4 = 1 } mxn_scale_layout;
+
+/* Bytes a scale buffer needs for T rows of K scales in the given layout
+ * (T*K row-major; ceil(T/128)*ceil(K/4)*512 tiled).  Returns 0 for a bad layout. */
+size_t mxn_scale_bytes(int64_t T, int64_t K, mxn_scale_layout layout);
+
+const char* mxn_status_string(mxn_status s);
+
+/* MXCast - Section 3.2 "Conversion to MXFP8", Eqs. S_tk = cast(m_tk / 256; E8M0),
+ * V_tkb = cast(X_tkb / S_tk; E4M3).
+ *   x_bf16 [T,D] in; codes_u8 [T,D] out; scales_u8 out (biased E8M0 exponents;
+ *   a zero block gets 0). */
+mxn_status mx_cast(const void* x_bf16, int64_t T, int64_t D, int block,
+                   void* codes_u8, void* scales_u8,
+                   mxn_round round, mxn_scale_layout layout, void* cuda_stream);
+
+/* Conventional path, fused - Algorithm 1 "RMSNorm + MXCast", Section 3.1 Eqs. rho_t, Y_td.
+ *   r_t = sqrt(mean_d x^2 + eps), rho = 1/r, y = x*rho (then *gain when gain_bf16 [D] is not
+ *   NULL), followed by MXCast of y without an intermediate bf16 rounding.
+ *   rms_out_or_null [T] fp32 receives r_t (what the backward consumes).
+ *   The mean of squares is accumulated in binary32 per thread and binary64 across threads:
+ *   r_t agrees with the binary64 definition to about 1e-7 relative, not bit for bit. */
+mxn_status rmsnorm_mxfp8_fwd(const void* x_bf16, const void* gain_bf16_or_null,
+                             int64_t T, int64_t D, int block, float eps,
+                             void* codes_u8, void* scales_u8, float* rms_out_or_null,
+                             mxn_round round, mxn_scale_layout layout, void* cuda_stream);
+
+/* MXNorm - Algorithm 2, Section 3.4 Eqs. m~_tk, rho~_t, S~_tk, V~_tkb.
+ *   m_k = block absmax of |x|; G = (1/K sum m_k^p)^(1/p), p in {1, 2};
+ *   r~ = coef * G (coef_or_0 == 0 selects the paper's printed constant for (B, p):
+ *   0.4185 for B = 32, p = 2); rho~ = 1 / (r~ + eps) (0 when the denominator is 0);
+ *   scales from m_k * rho~, codes from x * rho~ / S.
+ *   gain_bf16_or_null: NULL is the paper's path (the gain is folded into the next weight,
+ *   Section 3.7).  Non-NULL is an extension: rho~ still comes from |x|, but scales and codes
+ *   are taken from (x * rho~) * gain.
+ *   rms_est_out_or_null [T] fp32 receives r~ (cached for the backward, Section 3.7). */
+mxn_status mxnorm_fwd(const void* x_bf16, const void* gain_bf16_or_null,
+                      int64_t T, int64_t D, int block, int p, float coef_or_0, float eps,
+                      void* codes_u8, void* scales_u8, float* rms_est_out_or_null,
+                      mxn_round round, mxn_scale_layout layout, void* cuda_stream);
+
+/* NVFP4 variant of MXNorm (the paper benchmarks "B = 16, E2M1" in Section 4.3 but does not
+ * define the scale rule; this is the usual NVFP4 convention).
+ *   B = 16; r~ and rho~ as in mxnorm_fwd with the (16, p) constant (0.4688 for p = 2);
+ *   block scale = E4M3(m_k * rho~ / 6 * global_scale) stored as one E4M3 byte per block
+ *   ([T, D/16], row-major or tiled as above); codes = E2M1(x * rho~ * global_scale / scale),
+ *   two per byte, element 2i in the low nibble: codes_u8_packed [T, D/2], 8-byte aligned.
+ *   Dequantisation: value = code * scale / global_scale.  global_scale = 1 is safe because
+ *   MXNorm's output is bounded by sqrt(K)/coef (Lemma 2). */
+mxn_status mxnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D,
+                            int p, float coef_or_0, float eps, float global_scale,
+                            void* codes_u8_packed, void* scales_e4m3, float* rms_est_out_or_null,
+                            mxn_scale_layout layout, void* cuda_stream);
+
+/* Backward - appendix "RMSNorm gradients", used as a straight-through estimator for MXNorm
+ * (Section 3.7): the RMSNorm gradient evaluated with the r the forward saved (r~ from
+ * mxnorm_fwd, or the true RMS from rmsnorm_mxfp8_fwd - same formula).
+ *   grad_out_bf16 [T,D] = dL/dZ with Z = (X / r) * gain;
+ *   h = grad_out * gain; delta_t = mean_d(h * x);
+ *   dx = h / r - x * delta / r^3        -> dx [T,D], bf16 (dx_is_fp32 == 0) or fp32;
+ *   dgain_j = sum_t (x_tj / r_t) * grad_out_tj -> dgain_f32_or_null [D] fp32.
+ *   Row sums in binary32; the column sum is a deterministic two-stage reduction through
+ *   `workspace` (device memory, >= mxnorm_bwd_workspace_bytes(T, D) bytes, 16-byte aligned;
+ *   contents on entry irrelevant, clobbered on exit; may be NULL when dgain is NULL). */
+mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,
+                      const float* rms, int64_t T, int64_t D,
+                      void* dx, int dx_is_fp32, float* dgain_f32_or_null,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t mxnorm_bwd_workspace_bytes(int64_t T, int64_t D);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXNORM_H_ */
