@@ -137,6 +137,23 @@ mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void*
                       void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t mxnorm_bwd_workspace_bytes(int64_t T, int64_t D);
 
+/* End-to-end convenience for callers whose activations live in HOST memory: mxnorm_fwd (Algorithm 2,
+ * no gain) with the host<->device copies inside the call.
+ *   x_host_bf16 [T,D], codes_host [T,D], scales_host (mxn_scale_bytes), rms_est_host_or_null [T]
+ *   are HOST pointers (pinned memory for asynchronous copies; pageable memory works but serialises).
+ *   workspace is DEVICE memory of at least mxnorm_fwd_host_workspace_bytes(T, D, block, layout) bytes,
+ *   256-byte aligned, used as staging.  Rows are processed in chunks: the host-to-device copy of chunk
+ *   i+1, the kernel of chunk i and the device-to-host copy of chunk i-1 overlap on two internal
+ *   non-blocking streams (created on the first call on each device - make that call outside any
+ *   stream capture), ordered after prior work on `cuda_stream` and joined back into it.
+ *   The call returns once everything is enqueued; the outputs are valid after `cuda_stream` is
+ *   synchronised.  No device memory is allocated. */
+mxn_status mxnorm_fwd_host(const void* x_host_bf16, int64_t T, int64_t D, int block, int p, float coef_or_0,
+                           float eps, void* codes_host, void* scales_host, float* rms_est_host_or_null,
+                           mxn_round round, mxn_scale_layout layout,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t mxnorm_fwd_host_workspace_bytes(int64_t T, int64_t D, int block, mxn_scale_layout layout);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,0 +1,152 @@
+"""ctypes binding of libmxnorm.so: same names as the C ABI, argument marshalling only.
+
+Every step of the hot path runs in the CUDA kernels behind the C ABI; this module only turns
+torch CUDA tensors into device pointers and sizes.  There is no CPU fallback: if the compiled
+library is missing the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmxnorm.so")
+
+ROUND_RCEIL_POW2, ROUND_FLOOR_OCP, ROUND_RCEIL_MAX = 0, 1, 2
+SCALES_ROWMAJOR, SCALES_SWIZZLE_128x4 = 0, 1
+OK = 0
+
+EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd",
+           "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
+           "mxnorm_fwd_host_workspace_bytes")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2603_13180_b200.build` "
+        "(the MXNorm path has no fallback implementation)")
+
+lib = ctypes.CDLL(LIB_PATH)
+
+_vp, _i64, _i32, _f32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+lib.mxn_scale_bytes.argtypes = [_i64, _i64, _i32]
+lib.mxn_scale_bytes.restype = _sz
+lib.mxn_status_string.argtypes = [_i32]
+lib.mxn_status_string.restype = ctypes.c_char_p
+lib.mx_cast.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _i32, _vp]
+lib.rmsnorm_mxfp8_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
+lib.mxnorm_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
+lib.mxnorm_nvfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.mxnorm_bwd.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp, _sz, _vp]
+lib.mxnorm_bwd_workspace_bytes.argtypes = [_i64, _i64]
+lib.mxnorm_bwd_workspace_bytes.restype = _sz
+lib.mxnorm_fwd_host.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]
+lib.mxnorm_fwd_host_workspace_bytes.argtypes = [_i64, _i64, _i32, _i32]
+lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
+for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host"):
+    getattr(lib, _name).restype = _i32
+
+
+class MXNormError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def status_string(status: int) -> str:
+    return lib.mxn_status_string(status).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise MXNormError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def scale_bytes(T: int, K: int, layout: int = SCALES_ROWMAJOR) -> int:
+    return int(lib.mxn_scale_bytes(T, K, layout))
+
+
+def alloc_outputs(T: int, D: int, block: int = 32, layout: int = SCALES_ROWMAJOR, nvfp4: bool = False,
+                  device="cuda"):
+    """Allocates (codes, scales, rms) for one forward call (torch owns the memory)."""
+    codes = torch.empty((T, D // 2 if nvfp4 else D), dtype=torch.uint8, device=device)
+    scales = torch.empty((scale_bytes(T, D // block, layout),), dtype=torch.uint8, device=device)
+    rms = torch.empty((T,), dtype=torch.float32, device=device)
+    return codes, scales, rms
+
+
+def mx_cast(x, codes, scales, block=32, round=ROUND_RCEIL_POW2, layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mx_cast(_ptr(x), T, D, block, _ptr(codes), _ptr(scales), round, layout, _stream(stream)), "mx_cast")
+
+
+def rmsnorm_mxfp8_fwd(x, gain, codes, scales, rms_out=None, eps=0.0, block=32, round=ROUND_RCEIL_POW2,
+                      layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.rmsnorm_mxfp8_fwd(_ptr(x), _ptr(gain), T, D, block, eps, _ptr(codes), _ptr(scales), _ptr(rms_out),
+                                 round, layout, _stream(stream)), "rmsnorm_mxfp8_fwd")
+
+
+def mxnorm_fwd(x, gain, codes, scales, rms_est_out=None, p=2, coef=0.0, eps=0.0, block=32,
+               round=ROUND_RCEIL_POW2, layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mxnorm_fwd(_ptr(x), _ptr(gain), T, D, block, p, coef, eps, _ptr(codes), _ptr(scales),
+                          _ptr(rms_est_out), round, layout, _stream(stream)), "mxnorm_fwd")
+
+
+def mxnorm_nvfp4_fwd(x, codes_packed, scales_e4m3, rms_est_out=None, p=2, coef=0.0, eps=0.0, global_scale=1.0,
+                     layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mxnorm_nvfp4_fwd(_ptr(x), T, D, p, coef, eps, global_scale, _ptr(codes_packed), _ptr(scales_e4m3),
+                                _ptr(rms_est_out), layout, _stream(stream)), "mxnorm_nvfp4_fwd")
+
+
+def mxnorm_bwd_workspace_bytes(T: int, D: int) -> int:
+    return int(lib.mxnorm_bwd_workspace_bytes(T, D))
+
+
+def mxnorm_bwd(x, grad_out, gain, rms, dx, dgain=None, workspace=None, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    _dev(grad_out, torch.bfloat16, "grad_out")
+    T, D = x.shape
+    if dx.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("dx must be bf16 or fp32")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.mxnorm_bwd(_ptr(x), _ptr(grad_out), _ptr(gain), _ptr(rms), T, D, _ptr(dx),
+                          1 if dx.dtype == torch.float32 else 0, _ptr(dgain), _ptr(workspace), ws_bytes,
+                          _stream(stream)), "mxnorm_bwd")
+
+
+def mxnorm_fwd_host_workspace_bytes(T: int, D: int, block: int = 32, layout: int = SCALES_ROWMAJOR) -> int:
+    return int(lib.mxnorm_fwd_host_workspace_bytes(T, D, block, layout))
+
+
+def mxnorm_fwd_host(x_host, codes_host, scales_host, rms_est_host, workspace, p=2, coef=0.0, eps=0.0, block=32,
+                    round=ROUND_RCEIL_POW2, layout=SCALES_ROWMAJOR, stream=None):
+    """Host tensors in and out (pin them for asynchronous copies); `workspace` is a CUDA uint8 tensor."""
+    if x_host.is_cuda or codes_host.is_cuda or scales_host.is_cuda or x_host.dtype != torch.bfloat16:
+        raise ValueError("mxnorm_fwd_host takes host tensors (bf16 input)")
+    T, D = x_host.shape
+    _check(lib.mxnorm_fwd_host(_ptr(x_host), T, D, block, p, coef, eps, _ptr(codes_host), _ptr(scales_host),
+                               _ptr(rms_est_host), round, layout, _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream(stream)), "mxnorm_fwd_host")

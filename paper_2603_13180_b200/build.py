@@ -1,0 +1,44 @@
+"""Builds libmxnorm.so in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
+from __future__ import annotations
+
+import os
+import subprocess
+import sys
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+CSRC = os.path.join(_HERE, "csrc")
+LIB = os.path.join(_HERE, "libmxnorm.so")
+SOURCES = ["mxn_api.cu", "mxn_fwd.cu", "mxn_bwd.cu"]
+HEADERS = ["mxn_device.cuh", "mxn_internal.h", os.path.join("..", "..", "include", "mxnorm.h")]
+
+# No fast-math and no flush-to-zero: scale selection relies on IEEE division, subnormals and exact
+# power-of-two products.
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
+              "--ftz=false", "--prec-div=true", "--prec-sqrt=true",
+              "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
+
+
+def _stale() -> bool:
+    if not os.path.exists(LIB):
+        return True
+    t = os.path.getmtime(LIB)
+    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.abspath(__file__)]
+    return any(os.path.getmtime(d) > t for d in deps)
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    if force or _stale():
+        tmp = LIB + f".tmp{os.getpid()}"
+        cmd = ["nvcc", *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp,
+               *[os.path.join(CSRC, f) for f in SOURCES]]
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        if verbose:
+            sys.stderr.write(res.stderr)
+        if res.returncode != 0:
+            raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        os.replace(tmp, LIB)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -1,0 +1,141 @@
+// Device helpers shared by the libmxnorm kernels (sm_100a only).
+//
+// Arithmetic rules used throughout: every product that the contract calls "one IEEE binary32
+// operation" is written with an explicit round-to-nearest intrinsic so that the compiler cannot
+// contract or reassociate it; no flush-to-zero, no fast-math.
+#pragma once
+
+#include <cuda_fp4.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mxnorm.h"
+
+namespace mxn {
+
+constexpr int kWarp = 32;
+
+// ---- 256-bit global memory accesses (32 bytes per lane; address 32-byte aligned) ------------
+__device__ __forceinline__ void ld_v8(const void* p, uint32_t* r)
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void st_v8(void* p, const uint32_t* r)
+{
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void st_v4(void* p, const uint32_t* r)
+{
+    asm volatile("st.global.cs.v4.b32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+__device__ __forceinline__ void st_v2(void* p, const uint32_t* r)
+{
+    asm volatile("st.global.cs.v2.b32 [%0], {%1,%2};" :: "l"(p), "r"(r[0]), "r"(r[1]) : "memory");
+}
+
+// ---- bf16 pairs -----------------------------------------------------------------------------
+// max(|a|,|b|) per bf16 half; the sign bit of the result is the xor of the signs (ignored).
+__device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// the larger magnitude of the two halves of a bf16x2 word, as a binary32 (exact widening)
+__device__ __forceinline__ float hmax_abs_to_f32(uint32_t m2)
+{
+    uint32_t lo = (m2 << 16) & 0x7FFF0000u, hi = m2 & 0x7FFF0000u;
+    return __uint_as_float(lo > hi ? lo : hi);   // positive floats order like their bit patterns
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// ---- element casts --------------------------------------------------------------------------
+// two binary32 -> two E4M3 (RN-even, saturating to +-448); `lo` lands in the low byte
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
+{
+    uint16_t d;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ uint32_t cvt_e4m3x4(float e0, float e1, float e2, float e3)
+{
+    return cvt_e4m3x2(e0, e1) | (cvt_e4m3x2(e2, e3) << 16);
+}
+// two binary32 -> two E2M1 nibbles (RN-even, saturating to +-6); `lo` lands in the low nibble
+__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
+{
+    return __nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest);
+}
+// E4M3 byte (non-negative, finite) -> binary32, exact
+__device__ __forceinline__ float e4m3_to_f32(uint32_t c)
+{
+    uint32_t ef = (c >> 3) & 0xF, mf = c & 7;
+    // normal: (8+mf) * 2^(ef-10); subnormal: mf * 2^-9
+    return ef ? __uint_as_float(((ef + 120u) << 23) | (mf << 20)) : (float)mf * 0.001953125f;
+}
+
+// ---- E8M0 block scale -----------------------------------------------------------------------
+// biased exponent sb of the power-of-two scale S = 2^(sb-127) for a block whose (normalised)
+// absmax is a >= 0; element format E4M3 (largest power of two 2^8, largest value 448).
+__device__ __forceinline__ uint32_t e8m0_scale(float a, int round)
+{
+    uint32_t u = __float_as_uint(a);
+    uint32_t E = u >> 23, frac = u & 0x7FFFFFu;
+    if (E >= 255u) return frac ? 0u : 254u;      // not finite (outside the contract): NaN -> 0, Inf -> largest scale
+    int sb;
+    if (round == MXN_ROUND_RCEIL_POW2) {
+        sb = (int)E + (frac != 0) - 8;           // ceil(log2 a) - 8 + 127; E == 0 (zero/subnormal) clamps to 0
+    } else if (round == MXN_ROUND_FLOOR_OCP) {
+        sb = (int)E - 8;                         // floor(log2 a) - 8 + 127
+    } else {
+        uint32_t t = __float_as_uint(__fdiv_rn(a, 448.0f));
+        uint32_t Et = t >> 23;
+        sb = Et ? (int)Et + ((t & 0x7FFFFFu) != 0) : (t > 0x00400000u);   // subnormal quotient: 2^-127 < t -> 1
+    }
+    return (uint32_t)max(sb, 0);
+}
+// 2^(127-sb) as binary32 (sb = 254 gives the subnormal 2^-127)
+__device__ __forceinline__ float inv_scale(uint32_t sb)
+{
+    return __uint_as_float(sb >= 254u ? 0x00400000u : ((254u - sb) << 23));
+}
+__device__ __forceinline__ bool is_normal_f32(float f)
+{
+    uint32_t E = (__float_as_uint(f) >> 23) & 0xFFu;
+    return E != 0u && E != 255u;
+}
+
+// byte offset of scale (row, k) in the row-major or 128x4-tiled layout
+__device__ __forceinline__ int64_t scale_offset(int64_t row, int k, int K, int tiles_per_row, int layout)
+{
+    if (layout == MXN_SCALES_ROWMAJOR) return row * K + k;
+    int rr = (int)(row & 127);
+    return ((row >> 7) * tiles_per_row + (k >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (k & 3);
+}
+
+// ---- reductions -----------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+// barrier among the `nthreads` threads of one row group (ids 1..15; 0 is __syncthreads)
+__device__ __forceinline__ void group_barrier(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(nthreads) : "memory");
+}
+
+}  // namespace mxn

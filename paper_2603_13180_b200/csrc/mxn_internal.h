@@ -1,0 +1,47 @@
+// Host-side declarations shared by the libmxnorm translation units (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mxn {
+
+enum { STAT_NONE = 0, STAT_RMS = 1, STAT_MX = 2 };
+
+struct FwdParams {
+    const uint16_t* x;      // bf16 [T, D]
+    const uint16_t* gain;   // bf16 [D] or nullptr
+    uint8_t* codes;         // [T, D] (E4M3) or [T, D/2] (E2M1 pairs)
+    uint8_t* scales;        // row-major [T, K] or 128x4-tiled
+    float* rms_out;         // [T] or nullptr
+    int64_t T;
+    int D, K;
+    int p;
+    float coef, eps, global_scale;
+    int round, layout;
+    // filled by the launcher
+    int wpr, npass, rows_per_cta, tiles_per_row;
+};
+
+bool fwd_shape_supported(int64_t D, int B);
+cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
+
+struct BwdParams {
+    const uint16_t* x;      // bf16 [T, D]
+    const uint16_t* g;      // bf16 [T, D]
+    const uint16_t* gain;   // bf16 [D] or nullptr
+    const float* rms;       // [T]
+    void* dx;               // bf16 or fp32 [T, D]
+    float* dgain;           // [D] or nullptr
+    float* partial;         // workspace [P, D] fp32
+    int64_t T;
+    int D;
+    int dx_is_fp32;
+    int parts;              // number of partial rows in the workspace (= CTAs of the main kernel)
+};
+
+bool bwd_shape_supported(int64_t D);
+int bwd_parts(int64_t T, int64_t D);
+cudaError_t launch_bwd(BwdParams P, cudaStream_t stream);
+
+}  // namespace mxn

@@ -1,0 +1,187 @@
+"""GPU parity: the CUDA forward kernels (through the C ABI) against the CPU oracle, element by
+element on the same seeded bf16 bits."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_13180_b200 import workloads as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_13180_b200 import binding as b
+    return b
+
+
+def rows(T, D, seed, outliers=True):
+    w = wl.Workload("t", T, D, seed=seed, outlier_frac=0.002 if outliers else 0.0, has_gain=True)
+    inp = wl.make_inputs(w)
+    return wl.bits(inp["x"]), wl.bits(inp["gain"])
+
+
+# shapes: single lane active, ragged K (not a multiple of 32), several passes, rows spanning
+# 2/4/8 warps, odd T (ragged last CTA)
+SHAPES = [(1, 32), (5, 64), (37, 768), (130, 1024), (9, 2560), (33, 4096), (6, 5120), (5, 8192), (3, 16384),
+          (2, 32768), (257, 2048)]
+
+
+@pytest.mark.parametrize("T,D", SHAPES)
+def test_mxnorm_fwd_matches_oracle_bit_for_bit(binding, oracle, T, D):
+    x, gain = rows(T, D, seed=T + D)
+    for p in (2, 1):
+        for eps in (0.0, 1e-5):
+            got = gu.run_fwd(binding, oracle, "mx", x, p=p, eps=eps)
+            gu.assert_exact(got, gu.run_ref(oracle, "mx", x, p=p, eps=eps), f"mxnorm p={p} eps={eps} {T}x{D}")
+    got = gu.run_fwd(binding, oracle, "mx", x, gain, eps=1e-5)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, eps=1e-5), f"mxnorm+gain {T}x{D}")
+    got = gu.run_fwd(binding, oracle, "mx", x, coef=0.5, eps=0.0)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, coef=0.5, eps=0.0), "mxnorm coef override")
+
+
+@pytest.mark.parametrize("T,D", SHAPES)
+def test_mx_cast_matches_oracle_bit_for_bit(binding, oracle, T, D):
+    x, _ = rows(T, D, seed=3 * T + D)
+    for rnd in (0, 1, 2):
+        got = gu.run_fwd(binding, oracle, "cast", x, round=rnd)
+        gu.assert_exact(got, gu.run_ref(oracle, "cast", x, round=rnd), f"mx_cast round={rnd} {T}x{D}")
+
+
+@pytest.mark.parametrize("T,D", SHAPES)
+def test_rmsnorm_mxfp8_fwd_matches_oracle(binding, oracle, T, D):
+    x, gain = rows(T, D, seed=5 * T + D)
+    for g in (None, gain):
+        got = gu.run_fwd(binding, oracle, "rms", x, g, eps=1e-5)
+        gu.assert_within_rounding_of_rho(got, gu.run_ref(oracle, "rms", x, g, eps=1e-5), 32, f"rmsnorm {T}x{D}")
+
+
+@pytest.mark.parametrize("block", [16, 64])
+@pytest.mark.parametrize("T,D", [(3, 64), (19, 1024), (7, 4096), (4, 8192), (3, 16384)])
+def test_other_block_sizes(binding, oracle, T, D, block):
+    x, gain = rows(T, D, seed=T + D + block)
+    got = gu.run_fwd(binding, oracle, "mx", x, block=block, eps=1e-5)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, block=block, eps=1e-5), f"mxnorm B={block}")
+    got = gu.run_fwd(binding, oracle, "mx", x, block=block, p=1)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, block=block, p=1), f"mxnorm p=1 B={block}")
+    got = gu.run_fwd(binding, oracle, "cast", x, block=block)
+    gu.assert_exact(got, gu.run_ref(oracle, "cast", x, block=block), f"mx_cast B={block}")
+    got = gu.run_fwd(binding, oracle, "rms", x, gain, block=block, eps=1e-5)
+    gu.assert_within_rounding_of_rho(got, gu.run_ref(oracle, "rms", x, gain, block=block, eps=1e-5), block, "rms")
+
+
+@pytest.mark.parametrize("rnd", [1, 2])
+def test_other_rounding_modes(binding, oracle, rnd):
+    x, gain = rows(41, 2048, seed=17)
+    got = gu.run_fwd(binding, oracle, "mx", x, round=rnd, eps=1e-5)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, round=rnd, eps=1e-5), f"mxnorm round={rnd}")
+    got = gu.run_fwd(binding, oracle, "mx", x, gain, round=rnd)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, round=rnd), f"mxnorm gain round={rnd}")
+
+
+@pytest.mark.parametrize("T,D", [(1, 32), (37, 768), (128, 128), (200, 192), (300, 4096), (129, 2560)])
+def test_tiled_scale_layout(binding, oracle, T, D):
+    x, _ = rows(T, D, seed=T * 7 + D)
+    for kind in ("mx", "cast", "rms"):
+        got = gu.run_fwd(binding, oracle, kind, x, layout=1, eps=1e-5)
+        want = gu.run_ref(oracle, kind, x, eps=1e-5)
+        if kind == "rms":
+            gu.assert_within_rounding_of_rho(got, want, 32, "tiled rms")
+        else:
+            gu.assert_exact(got, want, f"tiled {kind} {T}x{D}")
+
+
+def test_all_bf16_bit_patterns(binding, oracle):
+    pats = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    pats = pats[(pats & 0x7F80) != 0x7F80]                      # finite values only
+    # as lone block maxima (mx_cast sees every exponent/mantissa, zeros, subnormals, the largest values) ...
+    x = np.zeros((pats.size, 64), np.uint16)
+    x[:, 0] = pats
+    x[:, 33] = pats >> 1
+    x[(x[:, 33] & 0x7F80) == 0x7F80, 33] = 0
+    for rnd in (0, 1, 2):
+        gu.assert_exact(gu.run_fwd(binding, oracle, "cast", x, round=rnd), gu.run_ref(oracle, "cast", x, round=rnd),
+                        f"patterns cast round={rnd}")
+    # ... and normalised: rows whose RMS estimate is far from 1 in both directions
+    rng = np.random.default_rng(0)
+    xr = pats[rng.integers(0, pats.size, size=(512, 256))]
+    xr[(xr & 0x7F80) > 0x5D00] &= 0x0FFF | 0x8000               # |x| < 2^60: squares stay inside binary32
+    for kind in ("mx", "rms"):
+        got = gu.run_fwd(binding, oracle, kind, xr)
+        want = gu.run_ref(oracle, kind, xr)
+        if kind == "mx":
+            gu.assert_exact(got, want, "random-pattern rows")
+        else:
+            gu.assert_within_rounding_of_rho(got, want, 32, "random-pattern rows rms")
+
+
+def test_degenerate_rows(binding, oracle):
+    D = 256
+    one = 0x3F80
+    x = np.zeros((8, D), np.uint16)
+    x[1, :] = 0x8000                      # all negative zeros
+    x[2, 5] = one                         # one-hot
+    x[3, :] = one                         # constant
+    x[4, :] = 0x0001                      # smallest subnormal everywhere
+    x[5, :] = 0x7F7F                      # largest finite everywhere
+    x[6, ::2] = 0x0080                    # smallest normal, alternating with zero
+    x[7, :32] = 0x7F00                    # one huge block, rest tiny
+    x[7, 32:] = 0x0100
+    for kind, exact in (("mx", True), ("cast", True), ("rms", False)):
+        got = gu.run_fwd(binding, oracle, kind, x)
+        want = gu.run_ref(oracle, kind, x)
+        if exact:
+            gu.assert_exact(got, want, f"degenerate {kind}")
+        else:
+            # rows 4-7 over/underflow a binary32 sum of squares: outside the baseline's stated domain
+            sel = [0, 1, 2, 3]
+            gu.assert_within_rounding_of_rho(tuple(a[sel] for a in got), tuple(a[sel] for a in want), 32, "degenerate rms")
+    got = gu.run_fwd(binding, oracle, "nvfp4", x[:, :256])
+    gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x[:, :256]), "degenerate nvfp4")
+    # constant-row closed form straight from the GPU: scale 121, code 0x72, r~ = fl32(0.4185)
+    codes, scales, r = gu.run_fwd(binding, oracle, "mx", x)
+    assert np.all(scales[3] == 121) and np.all(codes[3] == 0x72) and r.view(np.uint32)[3] == 0x3ED645A2
+
+
+@pytest.mark.parametrize("T,D", [(1, 16), (5, 48), (37, 768), (130, 1024), (33, 4096), (5, 8192), (3, 16384), (257, 2048)])
+def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
+    x, _ = rows(T, D, seed=11 * T + D)
+    for p, eps, gs in ((2, 1e-5, 1.0), (1, 0.0, 1.0), (2, 0.0, 8.0)):
+        got = gu.run_fwd(binding, oracle, "nvfp4", x, p=p, eps=eps, global_scale=gs)
+        gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x, p=p, eps=eps, global_scale=gs), f"nvfp4 {T}x{D} p={p}")
+    got = gu.run_fwd(binding, oracle, "nvfp4", x, layout=1)
+    gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x), "nvfp4 tiled scales")
+
+
+def test_power_of_two_shift_on_gpu(binding, oracle):
+    x, _ = rows(64, 1024, seed=23)
+    xv = (x.astype(np.uint32) << 16).view(np.float32)
+    base = gu.run_fwd(binding, oracle, "mx", x)
+    for k in (-9, 4):
+        xs = wl.f32_to_bf16_bits(xv * np.float32(2.0 ** k))
+        c, s, r = gu.run_fwd(binding, oracle, "mx", xs)
+        assert np.array_equal(c, base[0]) and np.array_equal(s, base[1])
+        assert np.array_equal(r, base[2] * np.float32(2.0 ** k))
+
+
+def test_runs_are_bitwise_repeatable(binding, oracle):
+    x, gain = rows(300, 4096, seed=29)
+    for kind in ("mx", "rms", "nvfp4"):
+        a = gu.run_fwd(binding, oracle, kind, x, eps=1e-5)
+        b = gu.run_fwd(binding, oracle, kind, x, eps=1e-5)
+        assert all(np.array_equal(u, v) for u, v in zip(a, b))
+
+
+def test_rms_output_is_optional_and_stream_is_honoured(binding, oracle):
+    x_bits, _ = rows(64, 1024, seed=31)
+    x = wl.from_bits(x_bits).cuda()
+    codes, scales, rms = binding.alloc_outputs(64, 1024)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        binding.mxnorm_fwd(x, None, codes, scales, None, eps=1e-5, stream=s)
+    s.synchronize()
+    want = gu.run_ref(oracle, "mx", x_bits, eps=1e-5)
+    assert np.array_equal(codes.cpu().numpy(), want[0]) and np.array_equal(scales.cpu().numpy().reshape(64, 32), want[1])
