@@ -17,13 +17,6 @@ def binding():
     return b
 
 
-def bf16_round_bits(oracle, a64):
-    flat = a64.ravel()
-    # vectorised RN-even of binary64 -> bf16 through exact binary32 when representable is not safe
-    # (double rounding), so use the oracle's direct rounding on the few values the test samples
-    return np.array([oracle.f64_to_bf16(float(v)) for v in flat], np.uint16).reshape(a64.shape)
-
-
 def bf16_ulp(v64):
     a = np.abs(v64)
     e = np.floor(np.log2(np.maximum(a, 2.0 ** -126)))
@@ -56,7 +49,11 @@ def check(binding, oracle, T, D, seed, with_gain=True):
     inp = wl.make_inputs(w)
     x, g = wl.bits(inp["x"]), wl.bits(inp["grad"])
     gain = wl.bits(inp["gain"]) if with_gain else None
-    _, _, rms = oracle.mxnorm_ref(x, eps=1e-5)
+    if D % 32 == 0:
+        _, _, rms = oracle.mxnorm_ref(x, eps=1e-5)            # the estimate the forward would save
+    else:                                                     # any positive r is a valid input of the backward
+        xv = (x.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        rms = (1.07 * np.sqrt((xv ** 2).mean(-1)) + 1e-5).astype(np.float32)
     want_dx, want_dg = oracle.mxnorm_bwd_ref(x, g, gain, rms)
     # fp32 output: per-row max-norm relative 1e-3 (binary32 row dot and products against binary64)
     dx, _, dg = run_bwd(binding, x, g, gain, rms, fp32_out=True)

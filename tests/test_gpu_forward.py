@@ -139,8 +139,10 @@ def test_degenerate_rows(binding, oracle):
             # rows 4-7 over/underflow a binary32 sum of squares: outside the baseline's stated domain
             sel = [0, 1, 2, 3]
             gu.assert_within_rounding_of_rho(tuple(a[sel] for a in got), tuple(a[sel] for a in want), 32, "degenerate rms")
-    got = gu.run_fwd(binding, oracle, "nvfp4", x[:, :256])
-    gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x[:, :256]), "degenerate nvfp4")
+    # NVFP4: row 6 (row scale 2^-126) makes rho~/scale overflow binary32, and 0 * Inf is a NaN whose sign is
+    # not defined: outside the stated domain (row scale within 2^+-100)
+    xs = x[[0, 1, 2, 3, 4, 5, 7]]
+    gu.assert_exact(gu.run_fwd(binding, oracle, "nvfp4", xs), gu.run_ref(oracle, "nvfp4", xs), "degenerate nvfp4")
     # constant-row closed form straight from the GPU: scale 121, code 0x72, r~ = fl32(0.4185)
     codes, scales, r = gu.run_fwd(binding, oracle, "mx", x)
     assert np.all(scales[3] == 121) and np.all(codes[3] == 0x72) and r.view(np.uint32)[3] == 0x3ED645A2
