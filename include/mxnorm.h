@@ -55,7 +55,8 @@ typedef enum {
     MXN_ERR_ENUM = 4,      /* unknown rounding mode / layout */
     MXN_ERR_WORKSPACE = 5, /* workspace NULL or smaller than the query says */
     MXN_ERR_CUDA = 6,      /* the CUDA runtime reported an error at launch */
-    MXN_ERR_TIMEOUT = 7    /* reserved: a bounded device-side wait ran out */
+    MXN_ERR_TIMEOUT = 7,   /* reserved: a bounded device-side wait ran out */
+    MXN_ERR_TOO_LARGE = 8  /* the problem needs more built-in scratch than the library holds */
 } mxn_status;
 
 /* Power-of-two rounding of the block scale (Section 3.2: "implementation-defined").
@@ -136,6 +137,27 @@ mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void*
                       void* dx, int dx_is_fp32, float* dgain_f32_or_null,
                       void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t mxnorm_bwd_workspace_bytes(int64_t T, int64_t D);
+
+/* mxnorm_bwd for callers that cannot provide a workspace (the paper has no counterpart; this is a
+ * convenience of this library).  Meant for code that may not allocate device memory where it runs:
+ * an op inside a framework's fixed memory plan, a plug-in that is handed only the op's tensors, a
+ * thread that must stay away from the allocator while another stream is being captured.
+ *   Same arguments and results as mxnorm_bwd minus the workspace.  The partial sums of dgain go to
+ *   an array built into the library's device image: mxnorm_bwd_noalloc_max_scratch_bytes() = 8 MiB,
+ *   reserved on every GPU that loads the library until the process exits.  The call needs
+ *   mxnorm_bwd_workspace_bytes(T, D) of it; if that is more (for example D = 16384 with T > 128),
+ *   it returns MXN_ERR_TOO_LARGE and enqueues nothing.  With dgain == NULL no scratch is used and any
+ *   supported size is accepted.
+ *   The first call on each device (with that device current) looks up the array's device address;
+ *   make that first call outside any stream capture.  No call allocates or frees memory.
+ *   All calls on a device share the one array.  It keeps whatever the previous call left; every
+ *   call rewrites the part it reads, so nothing has to be cleared.  Two calls whose kernels may
+ *   overlap on the GPU (different streams, no ordering between them) race on it and give wrong
+ *   dgain: order such calls, or use mxnorm_bwd with separate workspaces. */
+mxn_status mxnorm_bwd_noalloc(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,
+                              const float* rms, int64_t T, int64_t D,
+                              void* dx, int dx_is_fp32, float* dgain_f32_or_null, void* cuda_stream);
+size_t mxnorm_bwd_noalloc_max_scratch_bytes(void);
 
 /* End-to-end convenience for callers whose activations live in HOST memory: mxnorm_fwd (Algorithm 2,
  * no gain) with the host<->device copies inside the call.

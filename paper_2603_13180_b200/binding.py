@@ -20,7 +20,7 @@ OK = 0
 
 EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd",
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
-           "mxnorm_fwd_host_workspace_bytes")
+           "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -44,7 +44,11 @@ lib.mxnorm_bwd_workspace_bytes.restype = _sz
 lib.mxnorm_fwd_host.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]
 lib.mxnorm_fwd_host_workspace_bytes.argtypes = [_i64, _i64, _i32, _i32]
 lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
-for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host"):
+lib.mxnorm_bwd_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp]
+lib.mxnorm_bwd_noalloc_max_scratch_bytes.argtypes = []
+lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
+for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
+              "mxnorm_bwd_noalloc"):
     getattr(lib, _name).restype = _i32
 
 
@@ -150,3 +154,17 @@ def mxnorm_fwd_host(x_host, codes_host, scales_host, rms_est_host, workspace, p=
     _check(lib.mxnorm_fwd_host(_ptr(x_host), T, D, block, p, coef, eps, _ptr(codes_host), _ptr(scales_host),
                                _ptr(rms_est_host), round, layout, _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _stream(stream)), "mxnorm_fwd_host")
+
+
+def mxnorm_bwd_noalloc(x, grad_out, gain, rms, dx, dgain=None, stream=None):
+    """mxnorm_bwd for callers that cannot allocate a workspace: the dgain partial sums use an 8 MiB array
+    built into the library (shared by all calls on the device - do not overlap two calls).  Raises
+    MXNormError(MXN_ERR_TOO_LARGE) when the problem would need more scratch than that."""
+    _dev(x, torch.bfloat16, "x")
+    _dev(grad_out, torch.bfloat16, "grad_out")
+    T, D = x.shape
+    if dx.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("dx must be bf16 or fp32")
+    _check(lib.mxnorm_bwd_noalloc(_ptr(x), _ptr(grad_out), _ptr(gain), _ptr(rms), T, D, _ptr(dx),
+                                  1 if dx.dtype == torch.float32 else 0, _ptr(dgain), _stream(stream)),
+           "mxnorm_bwd_noalloc")

@@ -97,6 +97,7 @@ const char* mxn_status_string(mxn_status s)
         case MXN_ERR_WORKSPACE: return "workspace missing or too small";
         case MXN_ERR_CUDA: return "CUDA runtime error at launch";
         case MXN_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case MXN_ERR_TOO_LARGE: return "the problem needs more built-in scratch than the library holds";
         default: return "unknown status";
     }
 }

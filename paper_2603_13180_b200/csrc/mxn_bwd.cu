@@ -11,6 +11,8 @@
 // a second small kernel adds the rows in a fixed order (deterministic, no atomics).
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "mxn_device.cuh"
 #include "mxn_internal.h"
 
@@ -243,3 +245,84 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
 }
 
 }  // namespace mxn
+
+// ---- backward without any caller-provided scratch -------------------------------------------------
+//
+// Some callers of mxnorm_bwd cannot hand over a workspace because they cannot allocate device memory
+// at the point of the call: code running inside a framework's static memory plan, a plug-in that
+// only receives the tensors of the op, or a host thread that must not touch the allocator while
+// another stream is being captured.  For them the partial sums of dgamma live in a fixed array that
+// is part of this library's device image.  Every GPU that loads the library reserves it until the
+// process exits, so it is kept modest: 2 Mi floats = 8 MiB.
+namespace {
+
+constexpr size_t kNoAllocScratchFloats = size_t(2) << 20;
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchFloats];
+
+// In host code the name g_noalloc_scratch is only a handle for the symbol; the device address has
+// to be asked for once per device, with that device current.
+constexpr int kNoAllocMaxDevices = 64;
+float* g_noalloc_ptr[kNoAllocMaxDevices] = {};
+std::mutex g_noalloc_mutex;
+
+cudaError_t noalloc_scratch_for_current_device(float** out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        if (p == nullptr) return cudaErrorInvalidSymbol;
+        g_noalloc_ptr[dev] = static_cast<float*>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+inline bool noalloc_misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
+}  // namespace
+
+extern "C" size_t mxnorm_bwd_noalloc_max_scratch_bytes(void) { return kNoAllocScratchFloats * sizeof(float); }
+
+extern "C" mxn_status mxnorm_bwd_noalloc(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,
+                                         const float* rms, int64_t T, int64_t D, void* dx, int dx_is_fp32,
+                                         float* dgain_f32_or_null, void* cuda_stream)
+{
+    if (T < 0 || D <= 0 || !mxn::bwd_shape_supported(D)) return MXN_ERR_SHAPE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (T == 0) {
+        if (dgain_f32_or_null != nullptr &&
+            cudaMemsetAsync(dgain_f32_or_null, 0, sizeof(float) * (size_t)D, s) != cudaSuccess)
+            return MXN_ERR_CUDA;
+        return MXN_OK;
+    }
+    if (x_bf16 == nullptr || grad_out_bf16 == nullptr || rms == nullptr || dx == nullptr) return MXN_ERR_NULL;
+    if (noalloc_misaligned(x_bf16, 16) || noalloc_misaligned(grad_out_bf16, 16) || noalloc_misaligned(dx, 16) ||
+        noalloc_misaligned(rms, 4) || (gain_bf16_or_null != nullptr && noalloc_misaligned(gain_bf16_or_null, 16)) ||
+        (dgain_f32_or_null != nullptr && noalloc_misaligned(dgain_f32_or_null, 16)))
+        return MXN_ERR_ALIGN;
+    const int parts = mxn::bwd_parts(T, D);
+    // the same launch as mxnorm_bwd needs parts * D floats of scratch: refuse what does not fit
+    if (dgain_f32_or_null != nullptr && (size_t)parts * (size_t)D > kNoAllocScratchFloats) return MXN_ERR_TOO_LARGE;
+    float* scratch = nullptr;
+    if (dgain_f32_or_null != nullptr && noalloc_scratch_for_current_device(&scratch) != cudaSuccess)
+        return MXN_ERR_CUDA;
+    mxn::BwdParams P{};
+    P.x = static_cast<const uint16_t*>(x_bf16);
+    P.g = static_cast<const uint16_t*>(grad_out_bf16);
+    P.gain = static_cast<const uint16_t*>(gain_bf16_or_null);
+    P.rms = rms;
+    P.dx = dx;
+    P.dgain = dgain_f32_or_null;
+    P.partial = scratch;   // every one of the `parts` rows is fully rewritten by its CTA: nothing to clear
+    P.T = T;
+    P.D = (int)D;
+    P.dx_is_fp32 = dx_is_fp32 != 0;
+    P.parts = parts;
+    return mxn::launch_bwd(P, s) == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
+}
