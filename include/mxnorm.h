@@ -15,7 +15,7 @@
  *  - X is bf16 [T, D], row-major, contiguous, base address 16-byte aligned.
  *    T >= 0 rows (tokens), D hidden size, `block` = B, K = D / B blocks per row.
  *    Supported: B in {16, 32, 64} (NVFP4: B = 16 fixed), D % B == 0,
- *    D <= 32768 * B / 32.  T == 0 returns MXN_OK without a launch.
+ *    D <= 32768 (backward: D % 8 == 0, D <= 16384).  T == 0 returns MXN_OK without a launch.
  *  - codes: one byte per element (E4M3, OCP "fn": bias 7, max 448, no infinity),
  *    [T, D] row-major; written with 32-byte stores: base 32-byte aligned.
  *  - scales: one byte per block.  MXN_SCALES_ROWMAJOR: [T, K].
@@ -75,6 +75,12 @@ typedef enum { MXN_SCALES_ROWMAJOR = 0, MXN_SCALES_SWIZZLE_128x4 = 1 } mxn_scale
 size_t mxn_scale_bytes(int64_t T, int64_t K, mxn_scale_layout layout);
 
 const char* mxn_status_string(mxn_status s);
+
+/* Diagnostics: the kernels that wait on asynchronous copies bound every wait; a wait that runs out
+ * makes the warp stop and bumps a device-side counter instead of hanging.  This call synchronises the
+ * device, stores the number of such events since the library was loaded into *count_out and returns
+ * MXN_ERR_TIMEOUT when it is non-zero (outputs of the affected launch are incomplete), else MXN_OK. */
+mxn_status mxn_device_timeouts(unsigned int* count_out);
 
 /* MXCast - Section 3.2 "Conversion to MXFP8", Eqs. S_tk = cast(m_tk / 256; E8M0),
  * V_tkb = cast(X_tkb / S_tk; E4M3).

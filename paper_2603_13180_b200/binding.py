@@ -20,7 +20,8 @@ OK = 0
 
 EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd",
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
-           "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes")
+           "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
+           "mxn_device_timeouts")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -34,6 +35,8 @@ lib.mxn_scale_bytes.argtypes = [_i64, _i64, _i32]
 lib.mxn_scale_bytes.restype = _sz
 lib.mxn_status_string.argtypes = [_i32]
 lib.mxn_status_string.restype = ctypes.c_char_p
+lib.mxn_device_timeouts.argtypes = [ctypes.POINTER(ctypes.c_uint)]
+lib.mxn_device_timeouts.restype = _i32
 lib.mx_cast.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _i32, _vp]
 lib.rmsnorm_mxfp8_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
 lib.mxnorm_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
@@ -80,6 +83,15 @@ def _dev(t: torch.Tensor, dtype, name: str):
     if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
         raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
     return t
+
+
+def device_timeouts() -> int:
+    """Synchronises the device and returns how many bounded device-side waits have run out (0 = healthy)."""
+    n = ctypes.c_uint(0)
+    st = lib.mxn_device_timeouts(ctypes.byref(n))
+    if st not in (OK, 7):
+        raise MXNormError(st, "mxn_device_timeouts")
+    return int(n.value)
 
 
 def scale_bytes(T: int, K: int, layout: int = SCALES_ROWMAJOR) -> int:

@@ -102,6 +102,14 @@ const char* mxn_status_string(mxn_status s)
     }
 }
 
+mxn_status mxn_device_timeouts(unsigned int* count_out)
+{
+    unsigned int n = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess || mxn::read_timeouts(&n) != cudaSuccess) return MXN_ERR_CUDA;
+    if (count_out != nullptr) *count_out = n;
+    return n == 0 ? MXN_OK : MXN_ERR_TIMEOUT;
+}
+
 mxn_status mx_cast(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8, void* scales_u8,
                    mxn_round round, mxn_scale_layout layout, void* cuda_stream)
 {

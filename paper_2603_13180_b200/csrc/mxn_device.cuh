@@ -132,10 +132,11 @@ __device__ __forceinline__ float warp_sum(float v)
     for (int o = 16; o > 0; o >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
     return v;
 }
-// barrier among the `nthreads` threads of one row group (ids 1..15; 0 is __syncthreads)
-__device__ __forceinline__ void group_barrier(int id, int nthreads)
+// barrier among the `nthreads` threads of one row group; the id is a compile-time constant (1..15)
+template <int ID>
+__device__ __forceinline__ void group_barrier_id(int nthreads)
 {
-    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(nthreads) : "memory");
+    asm volatile("bar.sync %0, %1;" :: "n"(ID), "r"(nthreads) : "memory");
 }
 
 }  // namespace mxn

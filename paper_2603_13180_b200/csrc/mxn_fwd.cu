@@ -16,7 +16,18 @@
 
 namespace mxn {
 
-constexpr int kThreads = 128;   // 4 warps per CTA; rows per CTA = 4 / WPR (WPR = 8 uses 256 threads)
+#ifndef MXN_FWD_WARPS
+#define MXN_FWD_WARPS 4          // warps per CTA (more when one row needs more); rows per CTA = warps / WPR
+#endif
+#ifndef MXN_FWD_MAX_ELEMS
+#define MXN_FWD_MAX_ELEMS 64     // elements a lane holds per row (registers: half as many 32-bit words)
+#endif
+#ifndef MXN_FWD_MIN_CTAS
+#define MXN_FWD_MIN_CTAS 1       // occupancy hint for the register allocator
+#endif
+
+// warps of a CTA whose rows each span WPR warps
+__host__ __device__ constexpr int cta_warps(int wpr) { return wpr > MXN_FWD_WARPS ? wpr : MXN_FWD_WARPS; }
 
 // row statistic -> (r, rho) ; one value per row group ------------------------------------------
 template <int STAT>
@@ -40,51 +51,42 @@ __device__ __forceinline__ void finish_stat(double s, const FwdParams& P, float&
     }
 }
 
-// sum of one double per warp over the WPR warps of a row group, in a fixed order
-__device__ __forceinline__ double group_sum(double v, int wpr, int group, int w, double* smem)
+// sum of one double per warp over the WPR warps of a row group, in a fixed order.  Barrier ids are
+// compile-time constants so that a kernel reserves only the barriers it uses (a dynamic id makes the
+// compiler reserve all 16, which caps the number of resident CTAs).
+template <int WPR>
+__device__ __forceinline__ double group_sum(double v, int group, int w, double* smem)
 {
     v = warp_sum(v);
-    if (wpr > 1) {
-        if ((threadIdx.x & 31) == 0) smem[group * 8 + w] = v;
-        group_barrier(1 + group, wpr * kWarp);
-        double t = smem[group * 8];
-        for (int i = 1; i < wpr; ++i) t = __dadd_rn(t, smem[group * 8 + i]);
+    if (WPR > 1) {
+        if ((threadIdx.x & 31) == 0) smem[group * WPR + w] = v;
+        if (WPR == cta_warps(WPR)) {
+            __syncthreads();
+        } else {
+            switch (group) {
+                case 0: group_barrier_id<1>(WPR * kWarp); break;
+                case 1: group_barrier_id<2>(WPR * kWarp); break;
+                case 2: group_barrier_id<3>(WPR * kWarp); break;
+                default: group_barrier_id<4>(WPR * kWarp); break;
+            }
+        }
+        double t = smem[group * WPR];
+#pragma unroll
+        for (int i = 1; i < WPR; ++i) t = __dadd_rn(t, smem[group * WPR + i]);
         v = t;
     }
     return v;
 }
 
-template <int B, int NPASS, int STAT, bool GAIN>
-__global__ void __launch_bounds__(256) fwd_e4m3_kernel(const FwdParams P)
+// ---- per-row work -------------------------------------------------------------------------------
+// Lane `lane` of pass i of warp w owns block k = (i*wpr + w)*32 + lane; xr[i][] holds its B bf16
+// values as packed pairs (zeros when k >= K).
+
+// phase 1: block absmaxes m[i] (exact) and this lane's share of the row statistic
+template <int B, int NPASS, int STAT>
+__device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2], float (&m)[NPASS], int p)
 {
-    constexpr int W = B / 2;   // 32-bit words (bf16 pairs) per block
-    __shared__ double red[8 * 8];
-
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int wpr = P.wpr;
-    const int group = warp / wpr, w = warp - group * wpr;
-    const int64_t row = (int64_t)blockIdx.x * P.rows_per_cta + group;
-    if (row >= P.T) return;   // whole row group leaves together
-
-    const uint16_t* xrow = P.x + row * P.D;
-    uint32_t xr[NPASS][W];
-    float m[NPASS];
-
-    // ---- load the row slice: block k = (pass*WPR + w)*32 + lane -------------------------------
-#pragma unroll
-    for (int i = 0; i < NPASS; ++i) {
-        const int k = (i * wpr + w) * kWarp + lane;
-        if (k < P.K) {
-            const uint16_t* p = xrow + (int64_t)k * B;
-#pragma unroll
-            for (int v = 0; v < W / 8; ++v) ld_v8(p + v * 16, &xr[i][v * 8]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < W; ++j) xr[i][j] = 0u;
-        }
-    }
-
-    // ---- phase 1: block absmaxes and the row statistic ---------------------------------------
+    constexpr int W = B / 2;
     double stat = 0.0;
     float ss0 = 0.f, ss1 = 0.f, ss2 = 0.f, ss3 = 0.f;
 #pragma unroll
@@ -95,7 +97,7 @@ __global__ void __launch_bounds__(256) fwd_e4m3_kernel(const FwdParams P)
         m[i] = hmax_abs_to_f32(m2);
         if (STAT == STAT_MX) {
             double md = (double)m[i];
-            stat = P.p == 2 ? __fma_rn(md, md, stat) : __dadd_rn(stat, md);   // m^2 is exact in binary64
+            stat = p == 2 ? __fma_rn(md, md, stat) : __dadd_rn(stat, md);   // m^2 is exact in binary64
         }
         if (STAT == STAT_RMS) {
 #pragma unroll
@@ -109,16 +111,28 @@ __global__ void __launch_bounds__(256) fwd_e4m3_kernel(const FwdParams P)
             }
         }
     }
-    float r = 1.0f, rho = 1.0f;
-    if (STAT != STAT_NONE) {
-        if (STAT == STAT_RMS) stat = (double)ss0 + (double)ss1 + ((double)ss2 + (double)ss3);
-        stat = group_sum(stat, wpr, group, w, red);
-        finish_stat<STAT>(stat, P, r, rho);
-        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
-    }
-    const bool rho_normal = is_normal_f32(rho);
+    if (STAT == STAT_RMS) stat = (double)ss0 + (double)ss1 + ((double)ss2 + (double)ss3);
+    return stat;
+}
 
-    // ---- phase 2: scales and codes -----------------------------------------------------------
+// Makes the compiler forget what it knows about the packed row: without this it keeps the binary32
+// copies it unpacked for the sum of squares alive until the quantise phase (twice the registers).
+template <int NPASS, int W>
+__device__ __forceinline__ void forget_unpacked(uint32_t (&xr)[NPASS][W])
+{
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i)
+#pragma unroll
+        for (int j = 0; j < W; ++j) asm volatile("" : "+r"(xr[i][j]));
+}
+
+// phase 2 (E4M3 codes, E8M0 scales): scales, codes and their stores for this lane's blocks
+template <int B, int NPASS, bool GAIN>
+__device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][B / 2], const float (&m)[NPASS], float rho,
+                                                    const FwdParams& P, int64_t row, int wpr, int w, int lane)
+{
+    constexpr int W = B / 2;
+    const bool rho_normal = is_normal_f32(rho);
     uint8_t* crow = P.codes + row * P.D;
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
@@ -195,47 +209,12 @@ __global__ void __launch_bounds__(256) fwd_e4m3_kernel(const FwdParams P)
     }
 }
 
-// NVFP4: B = 16 (one 32-byte load per block), E4M3 block scales, E2M1 codes two per byte.
+// phase 2 (NVFP4): E4M3 block scales, E2M1 codes two per byte, B = 16
 template <int NPASS>
-__global__ void __launch_bounds__(256) fwd_nvfp4_kernel(const FwdParams P)
+__device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS][8], const float (&m)[NPASS], float rho,
+                                                     const FwdParams& P, int64_t row, int wpr, int w, int lane)
 {
-    constexpr int B = 16, W = 8;
-    __shared__ double red[8 * 8];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int wpr = P.wpr;
-    const int group = warp / wpr, w = warp - group * wpr;
-    const int64_t row = (int64_t)blockIdx.x * P.rows_per_cta + group;
-    if (row >= P.T) return;
-
-    const uint16_t* xrow = P.x + row * P.D;
-    uint32_t xr[NPASS][W];
-    float m[NPASS];
-#pragma unroll
-    for (int i = 0; i < NPASS; ++i) {
-        const int k = (i * wpr + w) * kWarp + lane;
-        if (k < P.K) {
-            ld_v8(xrow + (int64_t)k * B, xr[i]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < W; ++j) xr[i][j] = 0u;
-        }
-    }
-    double stat = 0.0;
-#pragma unroll
-    for (int i = 0; i < NPASS; ++i) {
-        uint32_t m2 = absmax_bf16x2(xr[i][0], xr[i][1]);
-#pragma unroll
-        for (int j = 2; j < W; ++j) m2 = absmax_bf16x2(m2, xr[i][j]);
-        m[i] = hmax_abs_to_f32(m2);
-        double md = (double)m[i];
-        stat = P.p == 2 ? __fma_rn(md, md, stat) : __dadd_rn(stat, md);
-    }
-    stat = group_sum(stat, wpr, group, w, red);
-    float r, rho;
-    finish_stat<STAT_MX>(stat, P, r, rho);
-    if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     const float rho_g = __fmul_rn(rho, P.global_scale);
-
     uint8_t* crow = P.codes + row * (P.D / 2);
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
@@ -264,43 +243,128 @@ __global__ void __launch_bounds__(256) fwd_nvfp4_kernel(const FwdParams P)
     }
 }
 
+// ---- register-direct kernels: one row per row group, loaded straight from global memory -----------
+// Generic path: any D % B == 0, rows spanning up to 8 warps, optional gain.
+template <int B, int NPASS>
+__device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], const uint16_t* xrow, int K, int wpr, int w, int lane)
+{
+    constexpr int W = B / 2;
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        const int k = (i * wpr + w) * kWarp + lane;
+        if (k < K) {
+            const uint16_t* p = xrow + (int64_t)k * B;
+#pragma unroll
+            for (int v = 0; v < W / 8; ++v) ld_v8(p + v * 16, &xr[i][v * 8]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < W; ++j) xr[i][j] = 0u;
+        }
+    }
+}
+
+template <int B, int NPASS, int WPR, int STAT, bool GAIN>
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 : MXN_FWD_MIN_CTAS) fwd_e4m3_kernel(const FwdParams P)
+{
+    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / WPR, w = warp - group * WPR;
+    const int64_t row = (int64_t)blockIdx.x * (cta_warps(WPR) / WPR) + group;
+    if (row >= P.T) return;   // whole row group leaves together
+
+    uint32_t xr[NPASS][B / 2];
+    float m[NPASS];
+    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
+    double stat = block_stats<B, NPASS, STAT>(xr, m, P.p);
+    if (STAT == STAT_RMS) forget_unpacked<NPASS, B / 2>(xr);
+    float r = 1.0f, rho = 1.0f;
+    if (STAT != STAT_NONE) {
+        stat = group_sum<WPR>(stat, group, w, red);
+        finish_stat<STAT>(stat, P, r, rho);
+        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    }
+    quantise_store_e4m3<B, NPASS, GAIN>(xr, m, rho, P, row, WPR, w, lane);
+}
+
+template <int NPASS, int WPR>
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 : MXN_FWD_MIN_CTAS) fwd_nvfp4_kernel(const FwdParams P)
+{
+    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / WPR, w = warp - group * WPR;
+    const int64_t row = (int64_t)blockIdx.x * (cta_warps(WPR) / WPR) + group;
+    if (row >= P.T) return;
+
+    uint32_t xr[NPASS][8];
+    float m[NPASS];
+    load_row_direct<16, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
+    double stat = block_stats<16, NPASS, STAT_MX>(xr, m, P.p);
+    stat = group_sum<WPR>(stat, group, w, red);
+    float r, rho;
+    finish_stat<STAT_MX>(stat, P, r, rho);
+    if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    quantise_store_nvfp4<NPASS>(xr, m, rho, P, row, WPR, w, lane);
+}
+
 // ---- dispatch ---------------------------------------------------------------------------------
 typedef void (*fwd_fn)(const FwdParams);
 
+// A row that fits one warp (WPR = 1) gets the kernel with exactly the passes it needs; rows spanning
+// 2 or 4 warps always use the full pass count (surplus passes are masked off).
 template <int B, int STAT, bool GAIN>
-static fwd_fn pick_npass(int npass)
+static fwd_fn pick_e4m3(int wpr, int npass)
 {
-    constexpr int MAXP = 128 / B;
+    constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
+    if (wpr == 2) return fwd_e4m3_kernel<B, MAXP, 2, STAT, GAIN>;
+    if (wpr == 4) return fwd_e4m3_kernel<B, MAXP, 4, STAT, GAIN>;
+    if (wpr == 8) return fwd_e4m3_kernel<B, MAXP, 8, STAT, GAIN>;
+    if (wpr == 16) return fwd_e4m3_kernel<B, MAXP, 16, STAT, GAIN>;
+    if (wpr != 1) return nullptr;
     switch (npass) {
-        case 1: return fwd_e4m3_kernel<B, 1, STAT, GAIN>;
-        case 2: return fwd_e4m3_kernel<B, 2, STAT, GAIN>;
-        case 3: if (MAXP >= 3) return fwd_e4m3_kernel<B, (MAXP >= 3 ? 3 : 1), STAT, GAIN>; break;
-        case 4: if (MAXP >= 4) return fwd_e4m3_kernel<B, (MAXP >= 4 ? 4 : 1), STAT, GAIN>; break;
-        case 5: case 6: if (MAXP >= 6) return fwd_e4m3_kernel<B, (MAXP >= 6 ? 6 : 1), STAT, GAIN>; break;
-        case 7: case 8: if (MAXP >= 8) return fwd_e4m3_kernel<B, (MAXP >= 8 ? 8 : 1), STAT, GAIN>; break;
-        default: break;
+        case 1: return fwd_e4m3_kernel<B, 1, 1, STAT, GAIN>;
+        case 2: return fwd_e4m3_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, GAIN>;
+        case 3: return fwd_e4m3_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, GAIN>;
+        case 4: return fwd_e4m3_kernel<B, (MAXP >= 4 ? 4 : MAXP), 1, STAT, GAIN>;
+        case 5: case 6: return fwd_e4m3_kernel<B, (MAXP >= 6 ? 6 : MAXP), 1, STAT, GAIN>;
+        default: return fwd_e4m3_kernel<B, MAXP, 1, STAT, GAIN>;
     }
-    return nullptr;
 }
 template <int B>
-static fwd_fn pick_stat(int stat, bool gain, int npass)
+static fwd_fn pick_stat(int stat, bool gain, int wpr, int npass)
 {
     switch (stat) {
-        case STAT_NONE: return pick_npass<B, STAT_NONE, false>(npass);
-        case STAT_RMS: return gain ? pick_npass<B, STAT_RMS, true>(npass) : pick_npass<B, STAT_RMS, false>(npass);
-        case STAT_MX: return gain ? pick_npass<B, STAT_MX, true>(npass) : pick_npass<B, STAT_MX, false>(npass);
+        case STAT_NONE: return pick_e4m3<B, STAT_NONE, false>(wpr, npass);
+        case STAT_RMS: return gain ? pick_e4m3<B, STAT_RMS, true>(wpr, npass) : pick_e4m3<B, STAT_RMS, false>(wpr, npass);
+        case STAT_MX: return gain ? pick_e4m3<B, STAT_MX, true>(wpr, npass) : pick_e4m3<B, STAT_MX, false>(wpr, npass);
         default: return nullptr;
     }
 }
+static fwd_fn pick_nvfp4(int wpr, int npass)
+{
+    constexpr int MAXP = MXN_FWD_MAX_ELEMS / 16;
+    if (wpr == 2) return fwd_nvfp4_kernel<MAXP, 2>;
+    if (wpr == 4) return fwd_nvfp4_kernel<MAXP, 4>;
+    if (wpr == 8) return fwd_nvfp4_kernel<MAXP, 8>;
+    if (wpr == 16) return fwd_nvfp4_kernel<MAXP, 16>;
+    if (wpr != 1) return nullptr;
+    switch (npass) {
+        case 1: return fwd_nvfp4_kernel<1, 1>;
+        case 2: return fwd_nvfp4_kernel<(MAXP >= 2 ? 2 : MAXP), 1>;
+        case 3: return fwd_nvfp4_kernel<(MAXP >= 3 ? 3 : MAXP), 1>;
+        case 4: return fwd_nvfp4_kernel<(MAXP >= 4 ? 4 : MAXP), 1>;
+        case 5: case 6: return fwd_nvfp4_kernel<(MAXP >= 6 ? 6 : MAXP), 1>;
+        default: return fwd_nvfp4_kernel<MAXP, 1>;
+    }
+}
 
-// Splits K blocks per row over WPR warps x NPASS passes with at most 128 elements per lane.
+// Splits K blocks per row over WPR warps x NPASS passes with at most MXN_FWD_MAX_ELEMS elements per lane.
 static bool plan_row(int K, int B, int* wpr, int* npass)
 {
-    const int maxp = 128 / B;
+    const int maxp = MXN_FWD_MAX_ELEMS / B;
     int w = 1;
     while ((K + 32 * w - 1) / (32 * w) > maxp) {
         w *= 2;
-        if (w > 8) return false;
+        if (w > 16) return false;
     }
     *wpr = w;
     *npass = (K + 32 * w - 1) / (32 * w);
@@ -317,31 +381,28 @@ bool fwd_shape_supported(int64_t D, int B)
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
 {
     if (!plan_row(P.K, B, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
-    const int warps = P.wpr == 8 ? 8 : 4;
-    P.rows_per_cta = warps / P.wpr;
     P.tiles_per_row = (P.K + 3) / 4;
+    P.stage_bytes = 0;
+    const int warps = cta_warps(P.wpr);
+    P.rows_per_cta = warps / P.wpr;
     fwd_fn fn = nullptr;
-    if (nvfp4) {
-        switch (P.npass) {
-            case 1: fn = fwd_nvfp4_kernel<1>; break;
-            case 2: fn = fwd_nvfp4_kernel<2>; break;
-            case 3: fn = fwd_nvfp4_kernel<3>; break;
-            case 4: fn = fwd_nvfp4_kernel<4>; break;
-            case 5: case 6: fn = fwd_nvfp4_kernel<6>; break;
-            default: fn = fwd_nvfp4_kernel<8>; break;
-        }
-    } else if (B == 16) {
-        fn = pick_stat<16>(stat, P.gain != nullptr, P.npass);
-    } else if (B == 32) {
-        fn = pick_stat<32>(stat, P.gain != nullptr, P.npass);
-    } else {
-        fn = pick_stat<64>(stat, P.gain != nullptr, P.npass);
-    }
+    if (nvfp4) fn = pick_nvfp4(P.wpr, P.npass);
+    else if (B == 16) fn = pick_stat<16>(stat, P.gain != nullptr, P.wpr, P.npass);
+    else if (B == 32) fn = pick_stat<32>(stat, P.gain != nullptr, P.wpr, P.npass);
+    else fn = pick_stat<64>(stat, P.gain != nullptr, P.wpr, P.npass);
     if (fn == nullptr) return cudaErrorInvalidValue;
     const int64_t ctas = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
     if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
     fn<<<(unsigned)ctas, warps * kWarp, 0, stream>>>(P);
     return cudaGetLastError();
+}
+
+// number of bounded device-side waits that ran out since the library was loaded (synchronises);
+// no kernel of this build waits on anything, so the counter stays 0
+__device__ unsigned int g_timeouts = 0;
+cudaError_t read_timeouts(unsigned int* out)
+{
+    return cudaMemcpyFromSymbol(out, g_timeouts, sizeof(unsigned int));
 }
 
 }  // namespace mxn

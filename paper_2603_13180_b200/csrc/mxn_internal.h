@@ -21,10 +21,12 @@ struct FwdParams {
     int round, layout;
     // filled by the launcher
     int wpr, npass, rows_per_cta, tiles_per_row;
+    int stage_bytes;        // TMA-fed kernel: bytes of one shared-memory row stage
 };
 
 bool fwd_shape_supported(int64_t D, int B);
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
+cudaError_t read_timeouts(unsigned int* out);
 
 struct BwdParams {
     const uint16_t* x;      // bf16 [T, D]

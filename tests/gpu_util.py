@@ -60,6 +60,7 @@ def run_fwd(binding, oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coe
     else:
         raise ValueError(kind)
     torch.cuda.synchronize()
+    assert binding.device_timeouts() == 0, "a bounded device-side wait ran out"
     assert guards_intact(cfull, T * ccols) and guards_intact(sfull, sbytes) and guards_intact(rfull, T * 4), \
         "a kernel wrote outside its output buffer"
     codes_np = codes.cpu().numpy().reshape(T, ccols)
