@@ -104,8 +104,11 @@ const char* mxn_status_string(mxn_status s)
 
 mxn_status mxn_device_timeouts(unsigned int* count_out)
 {
-    unsigned int n = 0;
-    if (cudaDeviceSynchronize() != cudaSuccess || mxn::read_timeouts(&n) != cudaSuccess) return MXN_ERR_CUDA;
+    unsigned int n = 0, nb = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess || mxn::read_timeouts(&n) != cudaSuccess ||
+        mxn::read_timeouts_bwd(&nb) != cudaSuccess)
+        return MXN_ERR_CUDA;
+    n += nb;
     if (count_out != nullptr) *count_out = n;
     return n == 0 ? MXN_OK : MXN_ERR_TIMEOUT;
 }

@@ -6,9 +6,17 @@
 //   dgamma_j = sum_t (x_tj / r_t) g_tj
 //
 // Work decomposition: a CTA owns ALL columns (thread i owns 16-byte vectors i, i+n, i+2n, ...)
-// and walks over rows, two at a time, so the per-column partial sums of dgamma stay in
-// registers for the whole kernel.  Each CTA writes one row of partial sums to the workspace;
-// a second small kernel adds the rows in a fixed order (deterministic, no atomics).
+// and walks over rows blockIdx, blockIdx + grid, ..., so the per-column partial sums of dgamma stay
+// in registers for the whole kernel.  Because the CTA is resident for many rows, the rows are fed
+// through a ring of shared-memory stages: one thread asks the bulk-copy engine for the x and g rows
+// of iteration i+STAGES (two instructions per row, completion signalled on an mbarrier) while the
+// CTA works on iteration i, which keeps STAGES rows per CTA in flight.  Each thread reads back only
+// the vectors it owns.  One __syncthreads per row (the row dot product) doubles as the "stage is
+// free" signal.  Each CTA writes one row of partial sums to the workspace; a second small kernel
+// adds the rows in a fixed order (deterministic, no atomics).
+//
+// Every wait on an mbarrier is bounded; if one runs out the CTA stops and a device-side counter is
+// raised (mxn_device_timeouts()).
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -19,29 +27,82 @@
 namespace mxn {
 
 constexpr int kSMs = 148;          // B200
-constexpr int kBwdCtasPerSM = 3;
-constexpr int kBwdRows = 2;        // rows in flight per CTA iteration (1 when a thread owns 4 vectors)
 
-__device__ __forceinline__ uint4 ldg_nc_v4(const void* p)
-{
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
-    return r;
-}
+__device__ unsigned int g_bwd_timeouts = 0;
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// false when the barrier did not complete within the spin budget (of the order of a second)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy (no multicast); addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
 
-template <int V, int R, bool GAIN, bool DGAIN>
+constexpr int kBwdMaxStages = 8;
+
+template <int V, bool GAIN, bool DGAIN>
 __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
 {
-    __shared__ float red[R][16];
+    extern __shared__ __align__(128) uint8_t ring_raw[];
+    __shared__ uint64_t full[kBwdMaxStages];
+    __shared__ float red[2][16];
+    __shared__ int abort_flag;
+
     const int tid = threadIdx.x, n = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = n >> 5;
     const int nvec = P.D >> 3;
+    const int stages = P.stages;
+    const uint32_t row_bytes = (uint32_t)P.D * 2u, half = (uint32_t)P.stage_bytes / 2u;
+    const uint32_t ring = smem_u32(ring_raw), bar0 = smem_u32(full);
     const float invD = __fdiv_rn(1.0f, (float)P.D);
+    const int64_t stride = gridDim.x;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < stages; ++s) mbar_init(bar0 + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int s = 0; s < stages; ++s) {
+            const int64_t row = (int64_t)blockIdx.x + s * stride;
+            if (row < P.T) {
+                mbar_expect_tx(bar0 + 8 * s, 2 * row_bytes);
+                bulk_load(ring + s * P.stage_bytes, P.x + row * P.D, row_bytes, bar0 + 8 * s);
+                bulk_load(ring + s * P.stage_bytes + half, P.g + row * P.D, row_bytes, bar0 + 8 * s);
+            }
+        }
+    }
 
     uint32_t gam[V][4];   // gain kept as packed bf16 pairs
     float acc[V][8];
@@ -54,95 +115,94 @@ __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[v][j] = 0.0f;
     }
+    __syncthreads();   // barriers initialised before anyone waits on them
 
-    for (int64_t row0 = (int64_t)blockIdx.x * R; row0 < P.T; row0 += (int64_t)gridDim.x * R) {
-        uint4 xw[R][V], gw[R][V];
-        float inv_r[R];
+    uint32_t it = 0;
+    float r_next = P.rms[blockIdx.x];   // the row's RMS is fetched one iteration ahead (keeps the load off the critical path)
+    for (int64_t row = blockIdx.x; row < P.T; row += stride, ++it) {
+        const uint32_t s = it % (uint32_t)stages, parity = (it / (uint32_t)stages) & 1u;
+        const uint32_t stage = ring + s * P.stage_bytes;
+        const float r_row = r_next;
+        if (row + stride < P.T) r_next = P.rms[row + stride];
+        if (!mbar_wait_bounded(bar0 + 8 * s, parity)) abort_flag = 1;
+
+        uint4 xw[V], gw[V];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int64_t row = row0 + r;
-            const bool live = row < P.T;
-            inv_r[r] = live ? __fdiv_rn(1.0f, P.rms[row]) : 0.0f;
+        for (int v = 0; v < V; ++v) {
+            const int vi = tid + v * n;
+            if (vi < nvec) {
+                xw[v] = lds_v4(stage + (uint32_t)vi * 16u);
+                gw[v] = lds_v4(stage + half + (uint32_t)vi * 16u);
+            } else {
+                xw[v] = make_uint4(0, 0, 0, 0);
+                gw[v] = make_uint4(0, 0, 0, 0);
+            }
+        }
+        const float inv_r = __fdiv_rn(1.0f, r_row);
+
+        // row dot sum_d h*x and the dgamma partials
+        float d0 = 0.f, d1 = 0.f;
 #pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int vi = tid + v * n;
-                if (live && vi < nvec) {
-                    xw[r][v] = ldg_nc_v4(reinterpret_cast<const uint4*>(P.x + row * P.D) + vi);
-                    gw[r][v] = ldg_nc_v4(reinterpret_cast<const uint4*>(P.g + row * P.D) + vi);
-                } else {
-                    xw[r][v] = make_uint4(0, 0, 0, 0);
-                    gw[r][v] = make_uint4(0, 0, 0, 0);
+        for (int v = 0; v < V; ++v) {
+            const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
+            const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
+                const float g0 = bf16_lo(ga[j]), g1 = bf16_hi(ga[j]);
+                const float h0 = GAIN ? g0 * bf16_lo(gam[v][j]) : g0, h1 = GAIN ? g1 * bf16_hi(gam[v][j]) : g1;
+                d0 = fmaf(h0, x0, d0);
+                d1 = fmaf(h1, x1, d1);
+                if (DGAIN) {
+                    acc[v][2 * j] = fmaf(x0 * inv_r, g0, acc[v][2 * j]);
+                    acc[v][2 * j + 1] = fmaf(x1 * inv_r, g1, acc[v][2 * j + 1]);
                 }
             }
         }
-        // row dots sum_d h*x and the dgamma partials
-        float dot[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float d0 = 0.f, d1 = 0.f;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const uint32_t xa[4] = {xw[r][v].x, xw[r][v].y, xw[r][v].z, xw[r][v].w};
-                const uint32_t ga[4] = {gw[r][v].x, gw[r][v].y, gw[r][v].z, gw[r][v].w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
-                    const float g0 = bf16_lo(ga[j]), g1 = bf16_hi(ga[j]);
-                    const float h0 = GAIN ? g0 * bf16_lo(gam[v][j]) : g0, h1 = GAIN ? g1 * bf16_hi(gam[v][j]) : g1;
-                    d0 = fmaf(h0, x0, d0);
-                    d1 = fmaf(h1, x1, d1);
-                    if (DGAIN) {
-                        acc[v][2 * j] = fmaf(x0 * inv_r[r], g0, acc[v][2 * j]);
-                        acc[v][2 * j + 1] = fmaf(x1 * inv_r[r], g1, acc[v][2 * j + 1]);
-                    }
-                }
+        const float dot = warp_sum(d0 + d1);
+        if (lane == 0) red[it & 1][warp] = dot;
+        __syncthreads();   // row dot complete; every thread has read its part of the stage
+        if (abort_flag) {
+            if (tid == 0) atomicAdd(&g_bwd_timeouts, 1u);
+            return;
+        }
+        if (tid == 0) {
+            const int64_t next = row + (int64_t)stages * stride;
+            if (next < P.T) {
+                mbar_expect_tx(bar0 + 8 * s, 2 * row_bytes);
+                bulk_load(stage, P.x + next * P.D, row_bytes, bar0 + 8 * s);
+                bulk_load(stage + half, P.g + next * P.D, row_bytes, bar0 + 8 * s);
             }
-            dot[r] = warp_sum(d0 + d1);
         }
-        if (lane == 0) {
+        float t = red[it & 1][0];
+        for (int i = 1; i < nwarps; ++i) t += red[it & 1][i];
+        const float delta = t * invD;
+        const float c1 = inv_r, c2 = delta * inv_r * inv_r * inv_r;
+
 #pragma unroll
-            for (int r = 0; r < R; ++r) red[r][warp] = dot[r];
-        }
-        __syncthreads();
-        float c1[R], c2[R];
+        for (int v = 0; v < V; ++v) {
+            const int vi = tid + v * n;
+            if (vi >= nvec) continue;
+            const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
+            const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
+            float o[8];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float t = red[r][0];
-            for (int i = 1; i < nwarps; ++i) t += red[r][i];
-            const float delta = t * invD;
-            c1[r] = inv_r[r];
-            c2[r] = delta * inv_r[r] * inv_r[r] * inv_r[r];
-        }
-        __syncthreads();   // red[] is rewritten by the next iteration
+            for (int j = 0; j < 4; ++j) {
+                const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
+                const float g0 = bf16_lo(ga[j]), g1 = bf16_hi(ga[j]);
+                const float h0 = GAIN ? g0 * bf16_lo(gam[v][j]) : g0, h1 = GAIN ? g1 * bf16_hi(gam[v][j]) : g1;
+                o[2 * j] = fmaf(-x0, c2, h0 * c1);
+                o[2 * j + 1] = fmaf(-x1, c2, h1 * c1);
+            }
+            if (P.dx_is_fp32) {
+                float* dp = static_cast<float*>(P.dx) + row * P.D + (int64_t)vi * 8;
+                st_v4(dp, reinterpret_cast<const uint32_t*>(o));
+                st_v4(dp + 4, reinterpret_cast<const uint32_t*>(o + 4));
+            } else {
+                uint32_t pk[4];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int64_t row = row0 + r;
-            if (row >= P.T) continue;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int vi = tid + v * n;
-                if (vi >= nvec) continue;
-                const uint32_t xa[4] = {xw[r][v].x, xw[r][v].y, xw[r][v].z, xw[r][v].w};
-                const uint32_t ga[4] = {gw[r][v].x, gw[r][v].y, gw[r][v].z, gw[r][v].w};
-                float o[8];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
-                    const float g0 = bf16_lo(ga[j]), g1 = bf16_hi(ga[j]);
-                    const float h0 = GAIN ? g0 * bf16_lo(gam[v][j]) : g0, h1 = GAIN ? g1 * bf16_hi(gam[v][j]) : g1;
-                    o[2 * j] = fmaf(-x0, c2[r], h0 * c1[r]);
-                    o[2 * j + 1] = fmaf(-x1, c2[r], h1 * c1[r]);
-                }
-                if (P.dx_is_fp32) {
-                    float* dp = static_cast<float*>(P.dx) + row * P.D + (int64_t)vi * 8;
-                    st_v4(dp, reinterpret_cast<const uint32_t*>(o));
-                    st_v4(dp + 4, reinterpret_cast<const uint32_t*>(o + 4));
-                } else {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) pk[j] = pack_bf16x2(o[2 * j], o[2 * j + 1]);
-                    st_v4(static_cast<uint16_t*>(P.dx) + row * P.D + (int64_t)vi * 8, pk);
-                }
+                for (int j = 0; j < 4; ++j) pk[j] = pack_bf16x2(o[2 * j], o[2 * j + 1]);
+                st_v4(static_cast<uint16_t*>(P.dx) + row * P.D + (int64_t)vi * 8, pk);
             }
         }
     }
@@ -182,9 +242,12 @@ __global__ void __launch_bounds__(256) bwd_dgain_reduce_kernel(const float* __re
     }
 }
 
-static bool plan_bwd(int64_t D, int* threads, int* V)
+// threads per CTA, vectors per thread, ring stages and CTAs per SM for a row of D elements
+struct BwdPlan { int threads, V, stages, stage_bytes, ctas_per_sm; size_t smem; };
+
+static bool plan_bwd(int64_t D, BwdPlan* pl)
 {
-    if (D <= 0 || D % 8 != 0) return false;
+    if (D <= 0 || D % 8 != 0 || D > 16384) return false;
     const int64_t nvec = D / 8;
     int n = (int)(((nvec < 256 ? nvec : 256) + 31) / 32 * 32);
     int v = (int)((nvec + n - 1) / n);
@@ -192,56 +255,66 @@ static bool plan_bwd(int64_t D, int* threads, int* V)
         n = 512;
         v = (int)((nvec + n - 1) / n);
     }
-    if (v > 4) return false;   // D <= 16384
-    *threads = n;
-    *V = v <= 2 ? v : 4;
-    return true;
+    if (v > 4) return false;
+    pl->threads = n;
+    pl->V = v <= 2 ? v : 4;
+    pl->stage_bytes = 2 * (int)((D * 2 + 127) / 128 * 128);     // x row + g row
+    pl->ctas_per_sm = n <= 256 ? 2 : 1;
+    const int budget = (n <= 256 ? 100 : 200) * 1024;           // shared memory per CTA
+    int st = budget / pl->stage_bytes;
+    pl->stages = st < 2 ? 2 : (st > kBwdMaxStages ? kBwdMaxStages : st);
+    pl->smem = (size_t)pl->stages * pl->stage_bytes;
+    return pl->smem <= 220 * 1024;
 }
 
 bool bwd_shape_supported(int64_t D)
 {
-    int n, v;
-    return plan_bwd(D, &n, &v);
+    BwdPlan pl;
+    return plan_bwd(D, &pl);
 }
-
-static int bwd_rows(int V) { return V <= 2 ? kBwdRows : 1; }
 
 int bwd_parts(int64_t T, int64_t D)
 {
-    int threads, V;
-    if (!plan_bwd(D, &threads, &V)) return 0;
-    const int R = bwd_rows(V);
-    const int64_t iters = (T + R - 1) / R;
-    const int64_t cap = (int64_t)kSMs * kBwdCtasPerSM;
-    return (int)(iters < cap ? (iters < 1 ? 1 : iters) : cap);
+    BwdPlan pl;
+    if (!plan_bwd(D, &pl)) return 0;
+    const int64_t cap = (int64_t)kSMs * pl.ctas_per_sm;
+    return (int)(T < cap ? (T < 1 ? 1 : T) : cap);
 }
 
-template <int V, int R>
-static void launch_v(const BwdParams& P, int threads, cudaStream_t s)
+typedef void (*bwd_fn)(const BwdParams);
+
+template <int V>
+static bwd_fn pick_bwd(bool gain, bool dgain)
 {
-    const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
-    if (gain && dgain) bwd_kernel<V, R, true, true><<<P.parts, threads, 0, s>>>(P);
-    else if (gain) bwd_kernel<V, R, true, false><<<P.parts, threads, 0, s>>>(P);
-    else if (dgain) bwd_kernel<V, R, false, true><<<P.parts, threads, 0, s>>>(P);
-    else bwd_kernel<V, R, false, false><<<P.parts, threads, 0, s>>>(P);
+    if (gain && dgain) return bwd_kernel<V, true, true>;
+    if (gain) return bwd_kernel<V, true, false>;
+    if (dgain) return bwd_kernel<V, false, true>;
+    return bwd_kernel<V, false, false>;
 }
 
 cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
 {
-    int threads, V;
-    if (!plan_bwd(P.D, &threads, &V)) return cudaErrorInvalidValue;
-    switch (V) {
-        case 1: launch_v<1, kBwdRows>(P, threads, stream); break;
-        case 2: launch_v<2, kBwdRows>(P, threads, stream); break;
-        default: launch_v<4, 1>(P, threads, stream); break;
-    }
-    cudaError_t e = cudaGetLastError();
+    BwdPlan pl;
+    if (!plan_bwd(P.D, &pl)) return cudaErrorInvalidValue;
+    P.stages = pl.stages;
+    P.stage_bytes = pl.stage_bytes;
+    const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
+    bwd_fn fn = pl.V == 1 ? pick_bwd<1>(gain, dgain) : pl.V == 2 ? pick_bwd<2>(gain, dgain) : pick_bwd<4>(gain, dgain);
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (e != cudaSuccess) return e;
+    fn<<<P.parts, pl.threads, pl.smem, stream>>>(P);
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (P.dgain != nullptr) {
         bwd_dgain_reduce_kernel<<<(P.D + 31) / 32, 256, 0, stream>>>(P.partial, P.dgain, P.D, P.parts);
         e = cudaGetLastError();
     }
     return e;
+}
+
+cudaError_t read_timeouts_bwd(unsigned int* out)
+{
+    return cudaMemcpyFromSymbol(out, g_bwd_timeouts, sizeof(unsigned int));
 }
 
 }  // namespace mxn

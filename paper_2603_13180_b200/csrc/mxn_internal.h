@@ -40,10 +40,12 @@ struct BwdParams {
     int D;
     int dx_is_fp32;
     int parts;              // number of partial rows in the workspace (= CTAs of the main kernel)
+    int stages, stage_bytes; // shared-memory ring (filled by the launcher)
 };
 
 bool bwd_shape_supported(int64_t D);
 int bwd_parts(int64_t T, int64_t D);
 cudaError_t launch_bwd(BwdParams P, cudaStream_t stream);
+cudaError_t read_timeouts_bwd(unsigned int* out);
 
 }  // namespace mxn

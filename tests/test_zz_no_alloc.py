@@ -52,7 +52,7 @@ def test_noalloc_backward_matches_workspace_backward_twice_in_a_row():
         pytest.skip("no CUDA device")
     from paper_2603_13180_b200 import binding as mx
     assert mx.lib.mxnorm_bwd_noalloc_max_scratch_bytes() == 8 << 20
-    # first call: 444 partial rows of 4096 floats (7.3 MB of the 8 MiB); second: 50 partial rows, other data
+    # first call: 296 partial rows of 4096 floats (4.6 MiB of the 8 MiB); second: 100 partial rows, other data
     _close(*_both(mx, 1200, 4096, seed=1, out_dtype=torch.float32))
     _close(*_both(mx, 100, 4096, seed=2, out_dtype=torch.bfloat16))
     # and once more with the first shape, after the smaller call
