@@ -73,8 +73,15 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr)
 
 constexpr int kBwdMaxStages = 8;
 
-template <int V, bool GAIN, bool DGAIN>
-__global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
+#ifndef MXN_BWD_THREADS
+#define MXN_BWD_THREADS 256      // threads per CTA for rows that need more than one vector per thread
+#endif
+#ifndef MXN_BWD_CTAS
+#define MXN_BWD_CTAS 2           // resident CTAs per SM the register allocator and the ring size aim for
+#endif
+
+template <int V, int NT, bool GAIN, bool DGAIN>
+__global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) bwd_kernel(const BwdParams P)
 {
     extern __shared__ __align__(128) uint8_t ring_raw[];
     __shared__ uint64_t full[kBwdMaxStages];
@@ -116,6 +123,7 @@ __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
         for (int j = 0; j < 8; ++j) acc[v][j] = 0.0f;
     }
     __syncthreads();   // barriers initialised before anyone waits on them
+    if (DGAIN) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // lets the reduction kernel's launch overlap this kernel
 
     uint32_t it = 0;
     float r_next = P.rms[blockIdx.x];   // the row's RMS is fetched one iteration ahead (keeps the load off the critical path)
@@ -140,7 +148,9 @@ __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
         }
         const float inv_r = __fdiv_rn(1.0f, r_row);
 
-        // row dot sum_d h*x and the dgamma partials
+        // One pass over the thread's elements with  gi = g/r,  t = gi*gamma (= h/r):
+        //   dgamma += x*gi ;  dot += t*x  (= sum_d h x / r) ;  later  dX = t - x * (dot/(D r^2)).
+        float tt[V][8];
         float d0 = 0.f, d1 = 0.f;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
@@ -149,14 +159,16 @@ __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
-                const float g0 = bf16_lo(ga[j]), g1 = bf16_hi(ga[j]);
-                const float h0 = GAIN ? g0 * bf16_lo(gam[v][j]) : g0, h1 = GAIN ? g1 * bf16_hi(gam[v][j]) : g1;
-                d0 = fmaf(h0, x0, d0);
-                d1 = fmaf(h1, x1, d1);
+                const float gi0 = bf16_lo(ga[j]) * inv_r, gi1 = bf16_hi(ga[j]) * inv_r;
                 if (DGAIN) {
-                    acc[v][2 * j] = fmaf(x0 * inv_r, g0, acc[v][2 * j]);
-                    acc[v][2 * j + 1] = fmaf(x1 * inv_r, g1, acc[v][2 * j + 1]);
+                    acc[v][2 * j] = fmaf(x0, gi0, acc[v][2 * j]);
+                    acc[v][2 * j + 1] = fmaf(x1, gi1, acc[v][2 * j + 1]);
                 }
+                const float t0 = GAIN ? gi0 * bf16_lo(gam[v][j]) : gi0, t1 = GAIN ? gi1 * bf16_hi(gam[v][j]) : gi1;
+                tt[v][2 * j] = t0;
+                tt[v][2 * j + 1] = t1;
+                d0 = fmaf(t0, x0, d0);
+                d1 = fmaf(t1, x1, d1);
             }
         }
         const float dot = warp_sum(d0 + d1);
@@ -176,23 +188,18 @@ __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
         }
         float t = red[it & 1][0];
         for (int i = 1; i < nwarps; ++i) t += red[it & 1][i];
-        const float delta = t * invD;
-        const float c1 = inv_r, c2 = delta * inv_r * inv_r * inv_r;
+        const float c2 = t * invD * inv_r * inv_r;   // delta / r^3 with delta = (t * r) / D
 
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int vi = tid + v * n;
             if (vi >= nvec) continue;
             const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
-            const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
             float o[8];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
-                const float g0 = bf16_lo(ga[j]), g1 = bf16_hi(ga[j]);
-                const float h0 = GAIN ? g0 * bf16_lo(gam[v][j]) : g0, h1 = GAIN ? g1 * bf16_hi(gam[v][j]) : g1;
-                o[2 * j] = fmaf(-x0, c2, h0 * c1);
-                o[2 * j + 1] = fmaf(-x1, c2, h1 * c1);
+                o[2 * j] = fmaf(-bf16_lo(xa[j]), c2, tt[v][2 * j]);
+                o[2 * j + 1] = fmaf(-bf16_hi(xa[j]), c2, tt[v][2 * j + 1]);
             }
             if (P.dx_is_fp32) {
                 float* dp = static_cast<float*>(P.dx) + row * P.D + (int64_t)vi * 8;
@@ -221,24 +228,43 @@ __global__ void __launch_bounds__(512) bwd_kernel(const BwdParams P)
     }
 }
 
-// dgain[j] = sum over the workspace rows, fixed order: 8 warps take rows w, w+8, ..., then the
-// 8 warp sums are added 0..7.  One CTA per 32 columns.
-__global__ void __launch_bounds__(256) bwd_dgain_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dgain,
-                                                              int D, int parts)
+// dgain[j] = sum over the workspace rows, in a fixed order.  One CTA of 32 warps per 128 columns:
+// warp w adds rows w, w+32, w+64, ... (a lane holds 4 columns, all its loads are issued before the
+// first add), then the 32 warp sums are added 0..31.  Launched with programmatic stream
+// serialisation so that its launch latency hides behind the tail of the main kernel; it waits for the
+// main kernel's results with griddepcontrol.wait before the first load.
+constexpr int kReduceMaxRowsPerWarp = 10;   // 32 warps x 10 rows >= 296 partial rows
+
+__global__ void __launch_bounds__(1024) bwd_dgain_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dgain,
+                                                               int D, int parts)
 {
-    __shared__ float s[8][32];
+    __shared__ float4 s[32][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int col = blockIdx.x * 32 + lane;
-    float a = 0.0f;
-    if (col < D)
-        for (int p = warp; p < parts; p += 8) a += partial[(int64_t)p * D + col];
+    const int col = (blockIdx.x * 32 + lane) * 4;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float4 v[kReduceMaxRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kReduceMaxRowsPerWarp; ++i) {
+        const int p = warp + 32 * i;
+        v[i] = (col < D && p < parts) ? *reinterpret_cast<const float4*>(partial + (int64_t)p * D + col)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 a = v[0];
+#pragma unroll
+    for (int i = 1; i < kReduceMaxRowsPerWarp; ++i) { a.x += v[i].x; a.y += v[i].y; a.z += v[i].z; a.w += v[i].w; }
+    for (int p = warp + 32 * kReduceMaxRowsPerWarp; p < parts; p += 32) {   // more partial rows than expected: plain loop
+        if (col < D) {
+            const float4 q = *reinterpret_cast<const float4*>(partial + (int64_t)p * D + col);
+            a.x += q.x; a.y += q.y; a.z += q.z; a.w += q.w;
+        }
+    }
     s[warp][lane] = a;
     __syncthreads();
     if (warp == 0 && col < D) {
-        float t = s[0][lane];
+        float4 t = s[0][lane];
 #pragma unroll
-        for (int i = 1; i < 8; ++i) t += s[i][lane];
-        dgain[col] = t;
+        for (int i = 1; i < 32; ++i) { const float4 q = s[i][lane]; t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w; }
+        *reinterpret_cast<float4*>(dgain + col) = t;
     }
 }
 
@@ -249,9 +275,9 @@ static bool plan_bwd(int64_t D, BwdPlan* pl)
 {
     if (D <= 0 || D % 8 != 0 || D > 16384) return false;
     const int64_t nvec = D / 8;
-    int n = (int)(((nvec < 256 ? nvec : 256) + 31) / 32 * 32);
+    int n = (int)(((nvec < MXN_BWD_THREADS ? nvec : MXN_BWD_THREADS) + 31) / 32 * 32);
     int v = (int)((nvec + n - 1) / n);
-    if (v > 2) {   // wide rows: more threads before more vectors per thread
+    if (v > 4) {   // wide rows: more threads before more vectors per thread
         n = 512;
         v = (int)((nvec + n - 1) / n);
     }
@@ -259,8 +285,8 @@ static bool plan_bwd(int64_t D, BwdPlan* pl)
     pl->threads = n;
     pl->V = v <= 2 ? v : 4;
     pl->stage_bytes = 2 * (int)((D * 2 + 127) / 128 * 128);     // x row + g row
-    pl->ctas_per_sm = n <= 256 ? 2 : 1;
-    const int budget = (n <= 256 ? 100 : 200) * 1024;           // shared memory per CTA
+    pl->ctas_per_sm = n <= MXN_BWD_THREADS ? MXN_BWD_CTAS : 1;
+    const int budget = 200 * 1024 / pl->ctas_per_sm;            // shared memory per CTA
     int st = budget / pl->stage_bytes;
     pl->stages = st < 2 ? 2 : (st > kBwdMaxStages ? kBwdMaxStages : st);
     pl->smem = (size_t)pl->stages * pl->stage_bytes;
@@ -283,13 +309,13 @@ int bwd_parts(int64_t T, int64_t D)
 
 typedef void (*bwd_fn)(const BwdParams);
 
-template <int V>
+template <int V, int NT>
 static bwd_fn pick_bwd(bool gain, bool dgain)
 {
-    if (gain && dgain) return bwd_kernel<V, true, true>;
-    if (gain) return bwd_kernel<V, true, false>;
-    if (dgain) return bwd_kernel<V, false, true>;
-    return bwd_kernel<V, false, false>;
+    if (gain && dgain) return bwd_kernel<V, NT, true, true>;
+    if (gain) return bwd_kernel<V, NT, true, false>;
+    if (dgain) return bwd_kernel<V, NT, false, true>;
+    return bwd_kernel<V, NT, false, false>;
 }
 
 cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
@@ -299,15 +325,31 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     P.stages = pl.stages;
     P.stage_bytes = pl.stage_bytes;
     const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
-    bwd_fn fn = pl.V == 1 ? pick_bwd<1>(gain, dgain) : pl.V == 2 ? pick_bwd<2>(gain, dgain) : pick_bwd<4>(gain, dgain);
+    bwd_fn fn;
+    if (pl.threads > MXN_BWD_THREADS) fn = pick_bwd<4, 512>(gain, dgain);
+    else if (pl.V == 1) fn = pick_bwd<1, MXN_BWD_THREADS>(gain, dgain);
+    else if (pl.V == 2) fn = pick_bwd<2, MXN_BWD_THREADS>(gain, dgain);
+    else fn = pick_bwd<4, MXN_BWD_THREADS>(gain, dgain);
     cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
     fn<<<P.parts, pl.threads, pl.smem, stream>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (P.dgain != nullptr) {
-        bwd_dgain_reduce_kernel<<<(P.D + 31) / 32, 256, 0, stream>>>(P.partial, P.dgain, P.D, P.parts);
-        e = cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((P.D + 127) / 128));
+        cfg.blockDim = dim3(1024);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const float* partial = P.partial;
+        float* dgain = P.dgain;
+        int D = P.D, parts = P.parts;
+        e = cudaLaunchKernelEx(&cfg, bwd_dgain_reduce_kernel, partial, dgain, D, parts);
     }
     return e;
 }
