@@ -63,14 +63,27 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
     return d;
 }
+// four binary32 -> four E4M3 bytes in memory order
 __device__ __forceinline__ uint32_t cvt_e4m3x4(float e0, float e1, float e2, float e3)
 {
-    return cvt_e4m3x2(e0, e1) | (cvt_e4m3x2(e2, e3) << 16);
+    uint32_t d;
+    asm("{ .reg .b16 lo, hi; cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1; cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3; mov.b32 %0, {lo, hi}; }"
+        : "=r"(d) : "f"(e0), "f"(e1), "f"(e2), "f"(e3));
+    return d;
 }
 // two binary32 -> two E2M1 nibbles (RN-even, saturating to +-6); `lo` lands in the low nibble
 __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
 {
     return __nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest);
+}
+// eight binary32 -> eight E2M1 nibbles in memory order (element 0 in the low nibble of byte 0)
+__device__ __forceinline__ uint32_t cvt_e2m1x8(float e0, float e1, float e2, float e3, float e4, float e5, float e6, float e7)
+{
+    uint32_t d;
+    asm("{ .reg .b8 b0, b1, b2, b3; cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1; cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3; "
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5; cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7; mov.b32 %0, {b0, b1, b2, b3}; }"
+        : "=r"(d) : "f"(e0), "f"(e1), "f"(e2), "f"(e3), "f"(e4), "f"(e5), "f"(e6), "f"(e7));
+    return d;
 }
 // E4M3 byte (non-negative, finite) -> binary32, exact
 __device__ __forceinline__ float e4m3_to_f32(uint32_t c)
@@ -100,6 +113,15 @@ __device__ __forceinline__ uint32_t e8m0_scale(float a, int round)
     }
     return (uint32_t)max(sb, 0);
 }
+// the paper's rule only (round up a/256 to a power of two): sb = max(ceil(log2 a) - 8 + 127, 0)
+__device__ __forceinline__ uint32_t e8m0_scale_rceil_pow2(float a)
+{
+    const uint32_t u = __float_as_uint(a);
+    const uint32_t E = u >> 23;
+    if (E >= 255u) return (u & 0x7FFFFFu) ? 0u : 254u;   // not finite (outside the contract)
+    const int sb = (int)E + ((u & 0x7FFFFFu) != 0u) - 8;
+    return (uint32_t)max(sb, 0);
+}
 // 2^(127-sb) as binary32 (sb = 254 gives the subnormal 2^-127)
 __device__ __forceinline__ float inv_scale(uint32_t sb)
 {
@@ -109,14 +131,6 @@ __device__ __forceinline__ bool is_normal_f32(float f)
 {
     uint32_t E = (__float_as_uint(f) >> 23) & 0xFFu;
     return E != 0u && E != 255u;
-}
-
-// byte offset of scale (row, k) in the row-major or 128x4-tiled layout
-__device__ __forceinline__ int64_t scale_offset(int64_t row, int k, int K, int tiles_per_row, int layout)
-{
-    if (layout == MXN_SCALES_ROWMAJOR) return row * K + k;
-    int rr = (int)(row & 127);
-    return ((row >> 7) * tiles_per_row + (k >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (k & 3);
 }
 
 // ---- reductions -----------------------------------------------------------------------------

@@ -35,14 +35,15 @@ __device__ __forceinline__ void finish_stat(double s, const FwdParams& P, float&
 {
     if (STAT == STAT_MX) {
         // G = (1/K sum m^p)^(1/p); r~ = fl32(coef * G); rho~ = 1 / fl32(r~ + eps)
-        double mean = __ddiv_rn(s, (double)P.K);
+        // (division by a power of two is an exact scaling: same result, far fewer instructions)
+        double mean = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.K);
         double G = P.p == 2 ? __dsqrt_rn(mean) : mean;
         r = __double2float_rn(__dmul_rn((double)P.coef, G));
         float den = __fadd_rn(r, P.eps);
         rho = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
     } else if (STAT == STAT_RMS) {
         // r = fl32(sqrt(mean x^2 + eps)); rho = 1 / r
-        double ms = __ddiv_rn(s, (double)P.D);
+        double ms = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.D);
         r = __double2float_rn(__dsqrt_rn(__dadd_rn(ms, (double)P.eps)));
         rho = r == 0.0f ? 0.0f : __fdiv_rn(1.0f, r);
     } else {
@@ -126,24 +127,43 @@ __device__ __forceinline__ void forget_unpacked(uint32_t (&xr)[NPASS][W])
         for (int j = 0; j < W; ++j) asm volatile("" : "+r"(xr[i][j]));
 }
 
-// phase 2 (E4M3 codes, E8M0 scales): scales, codes and their stores for this lane's blocks
-template <int B, int NPASS, bool GAIN>
+// byte offset of this lane's first scale (pass 0) and the distance between passes
+template <int WPR>
+__device__ __forceinline__ void scale_addressing(const FwdParams& P, int64_t row, int w, int lane, int64_t& off0, int64_t& step)
+{
+    const int k0 = w * kWarp + lane;
+    if (P.layout == MXN_SCALES_ROWMAJOR) {
+        off0 = row * P.K + k0;
+        step = WPR * kWarp;
+    } else {
+        const int rr = (int)(row & 127);
+        off0 = ((row >> 7) * P.tiles_per_row + (k0 >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (k0 & 3);
+        step = (int64_t)WPR * (kWarp / 4) * 512;   // 32*WPR blocks further = 8*WPR tiles of 512 bytes
+    }
+}
+
+// phase 2 (E4M3 codes, E8M0 scales): scales, codes and their stores for this lane's blocks.
+// PAPER selects the paper's rounding rule at compile time (the common case); otherwise P.round decides.
+template <int B, int NPASS, int WPR, bool GAIN, bool PAPER>
 __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][B / 2], const float (&m)[NPASS], float rho,
-                                                    const FwdParams& P, int64_t row, int wpr, int w, int lane)
+                                                    const FwdParams& P, int64_t row, int w, int lane)
 {
     constexpr int W = B / 2;
     const bool rho_normal = is_normal_f32(rho);
-    uint8_t* crow = P.codes + row * P.D;
+    uint8_t* cp0 = P.codes + row * P.D + (int64_t)(w * kWarp + lane) * B;
+    int64_t soff, sstep;
+    scale_addressing<WPR>(P, row, w, lane, soff, sstep);
+    uint8_t* sp0 = P.scales + soff;
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
-        const int k = (i * wpr + w) * kWarp + lane;
+        const int k = (i * WPR + w) * kWarp + lane;
         const bool active = k < P.K;
         uint32_t out[W / 2];
         uint32_t sb;
         if (!GAIN) {
             // a = fl32(m * rho) is also the absmax of fl32(x * rho): rounding is monotone
             const float a = __fmul_rn(m[i], rho);
-            sb = e8m0_scale(a, P.round);
+            sb = PAPER ? e8m0_scale_rceil_pow2(a) : e8m0_scale(a, P.round);
             const float inv = inv_scale(sb);
             // q = fl32(x*rho) * 2^(127-sb).  When neither factor product leaves the normal range the
             // two roundings collapse into the single product x * (rho * 2^(127-sb)).
@@ -185,7 +205,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
                 const float y1 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), bf16_hi(gr[j]));
                 my = fmaxf(my, fmaxf(fabsf(y0), fabsf(y1)));
             }
-            sb = e8m0_scale(my, P.round);
+            sb = PAPER ? e8m0_scale_rceil_pow2(my) : e8m0_scale(my, P.round);
             const float inv = inv_scale(sb);
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
@@ -197,28 +217,31 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
             }
         }
         if (active) {
-            uint8_t* cp = crow + (int64_t)k * B;
+            uint8_t* cp = cp0 + (int64_t)i * (WPR * kWarp * B);
             if (B == 16) {
                 st_v4(cp, out);
             } else {
 #pragma unroll
                 for (int v = 0; v < W / 16; ++v) st_v8(cp + v * 32, &out[v * 8]);
             }
-            P.scales[scale_offset(row, k, P.K, P.tiles_per_row, P.layout)] = (uint8_t)sb;
+            sp0[i * sstep] = (uint8_t)sb;
         }
     }
 }
 
 // phase 2 (NVFP4): E4M3 block scales, E2M1 codes two per byte, B = 16
-template <int NPASS>
+template <int NPASS, int WPR>
 __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS][8], const float (&m)[NPASS], float rho,
-                                                     const FwdParams& P, int64_t row, int wpr, int w, int lane)
+                                                     const FwdParams& P, int64_t row, int w, int lane)
 {
     const float rho_g = __fmul_rn(rho, P.global_scale);
-    uint8_t* crow = P.codes + row * (P.D / 2);
+    uint8_t* cp0 = P.codes + row * (P.D / 2) + (int64_t)(w * kWarp + lane) * 8;
+    int64_t soff, sstep;
+    scale_addressing<WPR>(P, row, w, lane, soff, sstep);
+    uint8_t* sp0 = P.scales + soff;
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
-        const int k = (i * wpr + w) * kWarp + lane;
+        const int k = (i * WPR + w) * kWarp + lane;
         // block scale = E4M3(fl32(fl32(a/6) * global_scale)), a = fl32(m * rho~)
         const float a = __fmul_rn(m[i], rho);
         const float t = __fmul_rn(__fdiv_rn(a, 6.0f), P.global_scale);
@@ -228,17 +251,15 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
         uint32_t out[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            uint32_t word = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t xw = xr[i][h * 4 + j];
-                word |= cvt_e2m1x2(__fmul_rn(bf16_lo(xw), inv), __fmul_rn(bf16_hi(xw), inv)) << (8 * j);
-            }
-            out[h] = word;
+            const uint32_t* xw = &xr[i][h * 4];
+            out[h] = cvt_e2m1x8(__fmul_rn(bf16_lo(xw[0]), inv), __fmul_rn(bf16_hi(xw[0]), inv),
+                                __fmul_rn(bf16_lo(xw[1]), inv), __fmul_rn(bf16_hi(xw[1]), inv),
+                                __fmul_rn(bf16_lo(xw[2]), inv), __fmul_rn(bf16_hi(xw[2]), inv),
+                                __fmul_rn(bf16_lo(xw[3]), inv), __fmul_rn(bf16_hi(xw[3]), inv));
         }
         if (k < P.K) {
-            st_v2(crow + (int64_t)k * 8, out);
-            P.scales[scale_offset(row, k, P.K, P.tiles_per_row, P.layout)] = (uint8_t)sc;
+            st_v2(cp0 + (int64_t)i * (WPR * kWarp * 8), out);
+            sp0[i * sstep] = (uint8_t)sc;
         }
     }
 }
@@ -263,7 +284,7 @@ __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], co
     }
 }
 
-template <int B, int NPASS, int WPR, int STAT, bool GAIN>
+template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 : MXN_FWD_MIN_CTAS) fwd_e4m3_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
@@ -283,7 +304,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 :
         finish_stat<STAT>(stat, P, r, rho);
         if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     }
-    quantise_store_e4m3<B, NPASS, GAIN>(xr, m, rho, P, row, WPR, w, lane);
+    quantise_store_e4m3<B, NPASS, WPR, GAIN, PAPER>(xr, m, rho, P, row, w, lane);
 }
 
 template <int NPASS, int WPR>
@@ -303,7 +324,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 :
     float r, rho;
     finish_stat<STAT_MX>(stat, P, r, rho);
     if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
-    quantise_store_nvfp4<NPASS>(xr, m, rho, P, row, WPR, w, lane);
+    quantise_store_nvfp4<NPASS, WPR>(xr, m, rho, P, row, w, lane);
 }
 
 // ---- dispatch ---------------------------------------------------------------------------------
@@ -311,33 +332,36 @@ typedef void (*fwd_fn)(const FwdParams);
 
 // A row that fits one warp (WPR = 1) gets the kernel with exactly the passes it needs; rows spanning
 // 2 or 4 warps always use the full pass count (surplus passes are masked off).
-template <int B, int STAT, bool GAIN>
+template <int B, int STAT, bool GAIN, bool PAPER>
 static fwd_fn pick_e4m3(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr == 2) return fwd_e4m3_kernel<B, MAXP, 2, STAT, GAIN>;
-    if (wpr == 4) return fwd_e4m3_kernel<B, MAXP, 4, STAT, GAIN>;
-    if (wpr == 8) return fwd_e4m3_kernel<B, MAXP, 8, STAT, GAIN>;
-    if (wpr == 16) return fwd_e4m3_kernel<B, MAXP, 16, STAT, GAIN>;
+    if (wpr == 2) return fwd_e4m3_kernel<B, MAXP, 2, STAT, GAIN, PAPER>;
+    if (wpr == 4) return fwd_e4m3_kernel<B, MAXP, 4, STAT, GAIN, PAPER>;
+    if (wpr == 8) return fwd_e4m3_kernel<B, MAXP, 8, STAT, GAIN, PAPER>;
+    if (wpr == 16) return fwd_e4m3_kernel<B, MAXP, 16, STAT, GAIN, PAPER>;
     if (wpr != 1) return nullptr;
     switch (npass) {
-        case 1: return fwd_e4m3_kernel<B, 1, 1, STAT, GAIN>;
-        case 2: return fwd_e4m3_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, GAIN>;
-        case 3: return fwd_e4m3_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, GAIN>;
-        case 4: return fwd_e4m3_kernel<B, (MAXP >= 4 ? 4 : MAXP), 1, STAT, GAIN>;
-        case 5: case 6: return fwd_e4m3_kernel<B, (MAXP >= 6 ? 6 : MAXP), 1, STAT, GAIN>;
-        default: return fwd_e4m3_kernel<B, MAXP, 1, STAT, GAIN>;
+        case 1: return fwd_e4m3_kernel<B, 1, 1, STAT, GAIN, PAPER>;
+        case 2: return fwd_e4m3_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, GAIN, PAPER>;
+        case 3: return fwd_e4m3_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, GAIN, PAPER>;
+        default: return fwd_e4m3_kernel<B, MAXP, 1, STAT, GAIN, PAPER>;
     }
 }
-template <int B>
+template <int B, bool PAPER>
 static fwd_fn pick_stat(int stat, bool gain, int wpr, int npass)
 {
     switch (stat) {
-        case STAT_NONE: return pick_e4m3<B, STAT_NONE, false>(wpr, npass);
-        case STAT_RMS: return gain ? pick_e4m3<B, STAT_RMS, true>(wpr, npass) : pick_e4m3<B, STAT_RMS, false>(wpr, npass);
-        case STAT_MX: return gain ? pick_e4m3<B, STAT_MX, true>(wpr, npass) : pick_e4m3<B, STAT_MX, false>(wpr, npass);
+        case STAT_NONE: return pick_e4m3<B, STAT_NONE, false, PAPER>(wpr, npass);
+        case STAT_RMS: return gain ? pick_e4m3<B, STAT_RMS, true, PAPER>(wpr, npass) : pick_e4m3<B, STAT_RMS, false, PAPER>(wpr, npass);
+        case STAT_MX: return gain ? pick_e4m3<B, STAT_MX, true, PAPER>(wpr, npass) : pick_e4m3<B, STAT_MX, false, PAPER>(wpr, npass);
         default: return nullptr;
     }
+}
+template <int B>
+static fwd_fn pick_round(int round, int stat, bool gain, int wpr, int npass)
+{
+    return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, true>(stat, gain, wpr, npass) : pick_stat<B, false>(stat, gain, wpr, npass);
 }
 static fwd_fn pick_nvfp4(int wpr, int npass)
 {
@@ -351,8 +375,6 @@ static fwd_fn pick_nvfp4(int wpr, int npass)
         case 1: return fwd_nvfp4_kernel<1, 1>;
         case 2: return fwd_nvfp4_kernel<(MAXP >= 2 ? 2 : MAXP), 1>;
         case 3: return fwd_nvfp4_kernel<(MAXP >= 3 ? 3 : MAXP), 1>;
-        case 4: return fwd_nvfp4_kernel<(MAXP >= 4 ? 4 : MAXP), 1>;
-        case 5: case 6: return fwd_nvfp4_kernel<(MAXP >= 6 ? 6 : MAXP), 1>;
         default: return fwd_nvfp4_kernel<MAXP, 1>;
     }
 }
@@ -382,14 +404,17 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
 {
     if (!plan_row(P.K, B, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
-    P.stage_bytes = 0;
+    {
+        const int count = stat == STAT_RMS ? P.D : P.K;   // divisor of the row statistic
+        P.inv_count = (count & (count - 1)) == 0 ? 1.0 / (double)count : 0.0;
+    }
     const int warps = cta_warps(P.wpr);
     P.rows_per_cta = warps / P.wpr;
     fwd_fn fn = nullptr;
     if (nvfp4) fn = pick_nvfp4(P.wpr, P.npass);
-    else if (B == 16) fn = pick_stat<16>(stat, P.gain != nullptr, P.wpr, P.npass);
-    else if (B == 32) fn = pick_stat<32>(stat, P.gain != nullptr, P.wpr, P.npass);
-    else fn = pick_stat<64>(stat, P.gain != nullptr, P.wpr, P.npass);
+    else if (B == 16) fn = pick_round<16>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
+    else if (B == 32) fn = pick_round<32>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
+    else fn = pick_round<64>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
     if (fn == nullptr) return cudaErrorInvalidValue;
     const int64_t ctas = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
     if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;

@@ -21,7 +21,7 @@ struct FwdParams {
     int round, layout;
     // filled by the launcher
     int wpr, npass, rows_per_cta, tiles_per_row;
-    int stage_bytes;        // TMA-fed kernel: bytes of one shared-memory row stage
+    double inv_count;       // 1/K (MXNorm) or 1/D (RMSNorm) when that is a power of two (exact), else 0
 };
 
 bool fwd_shape_supported(int64_t D, int B);
