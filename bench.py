@@ -244,6 +244,15 @@ def main():
             torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
 
+    # the same launches with an event record between them: an event breaks the programmatic dependency, so
+    # each kernel starts only after the previous one has fully retired (no overlap of launch and tail)
+    def fwd_serialised(i):
+        fwd(i)
+        marker.record(stream)
+
+    marker = torch.cuda.Event()
+    ms_serial = time_launches(fwd_serialised, SETS, args.steps, args.warmup, stream)
+
     nbytes = algorithmic_bytes("mx", T, D)
     gbs_one = nbytes / (ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
@@ -254,7 +263,11 @@ def main():
         "config": {"workload": f"{WORKLOAD}: mxnorm_fwd bf16 [{T},{D}] per GPU (batch 4 x seq 4096, Llama-3-8B hidden), "
                                "outlier channels, MXFP8 E4M3 codes + E8M0 scales (B=32) in the 128x4 tiled GEMM layout, p=2",
                    "l2": f"inputs/outputs rotate over {SETS} buffer sets ({SETS * nbytes / 1e6:.0f} MB > 126 MB L2)",
+                   "launch": "back-to-back launches in one stream, as the library issues them: programmatic stream "
+                             "serialisation (each kernel waits for the previous one before its first memory access; launch "
+                             "latency overlaps the previous kernel's tail); event_between_launches_ms_per_step records an event after every launch",
                    "parallelism": f"rows sharded, no collective (x{world})"},
+        "event_between_launches_ms_per_step": ms_serial,
         "tokens_per_s": T * world / (ms * 1e-3),
         "gpu_launches": args.steps,
         "clocks": clocks,

@@ -26,6 +26,13 @@
  *      ((r/128) * ceil(K/4) + c/4) * 512 + (r%32) * 16 + ((r%128)/32) * 4 + c%4.
  *    The buffer must hold mxn_scale_bytes(T, K, layout) bytes; padding bytes are
  *    written as 0.
+ *  - Launch semantics: kernels are launched with programmatic stream serialisation.  Each kernel
+ *    waits, before its first memory access, until the preceding kernel of the stream has completed and
+ *    its writes are visible, so ordering and results are those of ordinary stream order; only the
+ *    launch latency of one kernel overlaps the tail of the previous one.  A kernel that FOLLOWS a
+ *    libmxnorm kernel and is itself launched with the programmatic attribute must do the same wait
+ *    (griddepcontrol.wait / cudaGridDependencySynchronize) before reading libmxnorm's outputs;
+ *    ordinary launches need nothing.
  *  - Outputs are fully overwritten.  Inputs must be finite; results for NaN/Inf
  *    inputs are unspecified (no fault).
  *  - Every function returns a status; nothing aborts, throws or prints.  Argument

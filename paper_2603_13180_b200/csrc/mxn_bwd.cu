@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
     const float invD = __fdiv_rn(1.0f, (float)P.D);
     const int64_t stride = gridDim.x;
 
+    pdl_prologue();
     if (tid == 0) {
         abort_flag = 0;
         for (int s = 0; s < stages; ++s) mbar_init(bar0 + 8 * s, 1);
@@ -123,7 +124,6 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
         for (int j = 0; j < 8; ++j) acc[v][j] = 0.0f;
     }
     __syncthreads();   // barriers initialised before anyone waits on them
-    if (DGAIN) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // lets the reduction kernel's launch overlap this kernel
 
     uint32_t it = 0;
     float r_next = P.rms[blockIdx.x];   // the row's RMS is fetched one iteration ahead (keeps the load off the critical path)
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(1024) bwd_dgain_reduce_kernel(const float* __r
     __shared__ float4 s[32][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int col = (blockIdx.x * 32 + lane) * 4;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    pdl_prologue();
     float4 v[kReduceMaxRowsPerWarp];
 #pragma unroll
     for (int i = 0; i < kReduceMaxRowsPerWarp; ++i) {
@@ -332,20 +332,22 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     else fn = pick_bwd<4, MXN_BWD_THREADS>(gain, dgain);
     cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    fn<<<P.parts, pl.threads, pl.smem, stream>>>(P);
-    e = cudaGetLastError();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P.parts);
+    cfg.blockDim = dim3((unsigned)pl.threads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, fn, P);
     if (e != cudaSuccess) return e;
     if (P.dgain != nullptr) {
-        cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)((P.D + 127) / 128));
         cfg.blockDim = dim3(1024);
         cfg.dynamicSmemBytes = 0;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
         const float* partial = P.partial;
         float* dgain = P.dgain;
         int D = P.D, parts = P.parts;

@@ -133,6 +133,19 @@ __device__ __forceinline__ bool is_normal_f32(float f)
     return E != 0u && E != 255u;
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialisation and starts with this
+// prologue: wait until the preceding kernel of the stream has completed and its writes are visible
+// (a no-op when that kernel was not launched early), then allow the following kernel to be scheduled
+// while this one is still running.  Memory is only touched after the wait, so results are the same as
+// with fully serialised launches; what overlaps is the launch latency and block scheduling of one
+// kernel with the tail of the previous one.
+__device__ __forceinline__ void pdl_prologue()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- reductions -----------------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v)
 {

@@ -291,6 +291,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 :
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * (cta_warps(WPR) / WPR) + group;
+    pdl_prologue();
     if (row >= P.T) return;   // whole row group leaves together
 
     uint32_t xr[NPASS][B / 2];
@@ -314,6 +315,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 :
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * (cta_warps(WPR) / WPR) + group;
+    pdl_prologue();
     if (row >= P.T) return;
 
     uint32_t xr[NPASS][8];
@@ -418,8 +420,18 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     if (fn == nullptr) return cudaErrorInvalidValue;
     const int64_t ctas = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
     if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    fn<<<(unsigned)ctas, warps * kWarp, 0, stream>>>(P);
-    return cudaGetLastError();
+    // Programmatic stream serialisation: the kernel may be scheduled while the previous kernel of the
+    // stream drains; it does not touch memory before that kernel has completed (pdl_prologue).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas);
+    cfg.blockDim = dim3(warps * kWarp);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, P);
 }
 
 // number of bounded device-side waits that ran out since the library was loaded (synchronises);
