@@ -30,15 +30,17 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2603_13180_b200 import sharding  # noqa: E402
 from paper_2603_13180_b200 import workloads as wl  # noqa: E402
 
 WORKLOAD = "C3"
 EPS = 1e-5
 SETS = 4            # rotating input/output buffer sets: 4 x 203 MB > 126 MB of L2
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one mxnorm_fwd launch at [16384, 4096] taken from
-# the committed ncu summary (profiles/); None until a capture exists
-NCU_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one mxnorm_fwd launch at [16384, 4096], from the
+# committed ncu summary profiles/mxnorm_fwd_c3_ncu_full.md (134.24 MB read + 38.17 MB written; the
+# rest of the 69.2 MB of output is still dirty in L2 when the kernel ends)
+NCU_TRAFFIC_BYTES = 172_416_768
 
 
 def algorithmic_bytes(kind: str, T: int, D: int) -> int:
@@ -231,10 +233,7 @@ def main():
     if dist is not None:
         dist.barrier()
     ms = time_launches(fwd, SETS, args.steps, args.warmup, stream)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = sharding.max_over_ranks(ms, device="cuda")
     # keep the GPU under load a little longer so that the 50 ms sampler sees it
     if rank == 0:
         t_end = time.time() + 0.5
@@ -273,7 +272,8 @@ def main():
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": gbs_one, "peak": peak, "unit": "GB/s", "frac": gbs_one / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_8TBs": gbs_one / 8000.0,
-                     "traffic": NCU_TRAFFIC_BYTES, "algorithmic_bytes": nbytes, "kernel": "fwd_e4m3_kernel<32,4,MX>"},
+                     "traffic": NCU_TRAFFIC_BYTES if T == w.T else None, "algorithmic_bytes": nbytes,
+                     "kernel": "fwd_e4m3_kernel<B=32,NPASS=2,WPR=2,STAT=MX>"},
     }
 
     if not args.skip_others:
@@ -335,10 +335,7 @@ def main():
 
         e2e_steps = max(3, min(args.steps, 20))
         ms_e2e = time_launches(e2e_step, 1, e2e_steps, 3, stream)
-        if dist is not None:
-            t = torch.tensor([ms_e2e], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = sharding.max_over_ranks(ms_e2e, device="cuda")
         result["e2e"] = {"value": nbytes * world / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms_e2e,
                          "steps": e2e_steps, "h2d_bytes_per_step": T * D * 2,
                          "d2h_bytes_per_step": T * D + shh.numel() + 4 * T,
@@ -346,10 +343,10 @@ def main():
 
         # ---- CPU oracle on this machine's host cores (rank 0, one GPU runs only) ----
         if rank == 0 and world == 1:
-            gbs_cpu, dt, threads = oracle_throughput(wl.bits(x_cpu), reps=3)
+            gbs_cpu, dt, threads = oracle_throughput(wl.bits(x_cpu), reps=20)
             result["cpu_baseline"] = {"value": gbs_cpu, "unit": "GB/s", "cores": threads, "kind": "oracle",
                                       "seconds_per_batch": dt,
-                                      "sample": f"3 passes of the full [{T},{D}] batch through mxnorm_ref (OpenMP over rows)"}
+                                      "sample": f"20 passes of the full [{T},{D}] batch through mxnorm_ref (plain C, OpenMP over rows)"}
 
     if rank == 0:
         print(json.dumps(result))

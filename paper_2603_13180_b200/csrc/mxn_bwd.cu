@@ -228,43 +228,38 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
     }
 }
 
-// dgain[j] = sum over the workspace rows, in a fixed order.  One CTA of 32 warps per 128 columns:
-// warp w adds rows w, w+32, w+64, ... (a lane holds 4 columns, all its loads are issued before the
-// first add), then the 32 warp sums are added 0..31.  Launched with programmatic stream
-// serialisation so that its launch latency hides behind the tail of the main kernel; it waits for the
-// main kernel's results with griddepcontrol.wait before the first load.
+// dgain[j] = sum over the workspace rows, in a fixed order.  One CTA of 32 warps per 32 columns
+// (D/32 CTAs): warp w adds rows w, w+32, w+64, ... (all its loads are issued before the first add),
+// then the 32 warp sums are added 0..31.  Launched with programmatic stream serialisation so that its
+// launch latency hides behind the tail of the main kernel; it waits for the main kernel's results
+// before the first load.
 constexpr int kReduceMaxRowsPerWarp = 10;   // 32 warps x 10 rows >= 296 partial rows
 
 __global__ void __launch_bounds__(1024) bwd_dgain_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dgain,
                                                                int D, int parts)
 {
-    __shared__ float4 s[32][32];
+    __shared__ float s[32][33];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int col = (blockIdx.x * 32 + lane) * 4;
+    const int col = blockIdx.x * 32 + lane;
     pdl_prologue();
-    float4 v[kReduceMaxRowsPerWarp];
+    float v[kReduceMaxRowsPerWarp];
 #pragma unroll
     for (int i = 0; i < kReduceMaxRowsPerWarp; ++i) {
         const int p = warp + 32 * i;
-        v[i] = (col < D && p < parts) ? *reinterpret_cast<const float4*>(partial + (int64_t)p * D + col)
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[i] = (col < D && p < parts) ? partial[(int64_t)p * D + col] : 0.0f;
     }
-    float4 a = v[0];
+    float a = v[0];
 #pragma unroll
-    for (int i = 1; i < kReduceMaxRowsPerWarp; ++i) { a.x += v[i].x; a.y += v[i].y; a.z += v[i].z; a.w += v[i].w; }
-    for (int p = warp + 32 * kReduceMaxRowsPerWarp; p < parts; p += 32) {   // more partial rows than expected: plain loop
-        if (col < D) {
-            const float4 q = *reinterpret_cast<const float4*>(partial + (int64_t)p * D + col);
-            a.x += q.x; a.y += q.y; a.z += q.z; a.w += q.w;
-        }
-    }
+    for (int i = 1; i < kReduceMaxRowsPerWarp; ++i) a += v[i];
+    if (col < D)
+        for (int p = warp + 32 * kReduceMaxRowsPerWarp; p < parts; p += 32) a += partial[(int64_t)p * D + col];   // more rows than expected
     s[warp][lane] = a;
     __syncthreads();
     if (warp == 0 && col < D) {
-        float4 t = s[0][lane];
+        float t = s[0][lane];
 #pragma unroll
-        for (int i = 1; i < 32; ++i) { const float4 q = s[i][lane]; t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w; }
-        *reinterpret_cast<float4*>(dgain + col) = t;
+        for (int i = 1; i < 32; ++i) t += s[i][lane];
+        dgain[col] = t;
     }
 }
 
@@ -345,7 +340,7 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     e = cudaLaunchKernelEx(&cfg, fn, P);
     if (e != cudaSuccess) return e;
     if (P.dgain != nullptr) {
-        cfg.gridDim = dim3((unsigned)((P.D + 127) / 128));
+        cfg.gridDim = dim3((unsigned)((P.D + 31) / 32));
         cfg.blockDim = dim3(1024);
         cfg.dynamicSmemBytes = 0;
         const float* partial = P.partial;
