@@ -27,7 +27,8 @@ namespace mxn {
 #endif
 
 // warps of a CTA whose rows each span WPR warps
-__host__ __device__ constexpr int cta_warps(int wpr) { return wpr > MXN_FWD_WARPS ? wpr : MXN_FWD_WARPS; }
+__host__ __device__ constexpr int rows_per_cta(int wpr) { return MXN_FWD_WARPS / wpr > 1 ? MXN_FWD_WARPS / wpr : 1; }
+__host__ __device__ constexpr int cta_warps(int wpr) { return wpr * rows_per_cta(wpr); }
 
 // row statistic -> (r, rho) ; one value per row group ------------------------------------------
 template <int STAT>
@@ -61,7 +62,7 @@ __device__ __forceinline__ double group_sum(double v, int group, int w, double* 
     v = warp_sum(v);
     if (WPR > 1) {
         if ((threadIdx.x & 31) == 0) smem[group * WPR + w] = v;
-        if (WPR == cta_warps(WPR)) {
+        if (rows_per_cta(WPR) == 1) {
             __syncthreads();
         } else {
             switch (group) {
@@ -285,12 +286,12 @@ __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], co
 }
 
 template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 : MXN_FWD_MIN_CTAS) fwd_e4m3_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m3_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
-    const int64_t row = (int64_t)blockIdx.x * (cta_warps(WPR) / WPR) + group;
+    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
     pdl_prologue();
     if (row >= P.T) return;   // whole row group leaves together
 
@@ -309,12 +310,12 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 :
 }
 
 template <int NPASS, int WPR>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 : MXN_FWD_MIN_CTAS) fwd_nvfp4_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvfp4_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
-    const int64_t row = (int64_t)blockIdx.x * (cta_warps(WPR) / WPR) + group;
+    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
     pdl_prologue();
     if (row >= P.T) return;
 
@@ -332,17 +333,47 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, WPR > MXN_FWD_WARPS ? 1 :
 // ---- dispatch ---------------------------------------------------------------------------------
 typedef void (*fwd_fn)(const FwdParams);
 
-// A row that fits one warp (WPR = 1) gets the kernel with exactly the passes it needs; rows spanning
-// 2 or 4 warps always use the full pass count (surplus passes are masked off).
+// The headline kernels (B = 32 or NVFP4, no gain, the paper's rounding rule) exist for every number of
+// warps per row in kFineWpr, so that hidden sizes of the form {3,5,7} * 2^r fill their lanes; the
+// other variants exist for power-of-two warps per row only.
+static const int kFineWpr[] = {1, 2, 3, 4, 5, 6, 7, 8, 16};
+static const int kCoarseWpr[] = {1, 2, 4, 8, 16};
+
+template <int B, int NPASS, int STAT, bool GAIN, bool PAPER, bool FINE>
+static fwd_fn e4m3_by_wpr(int wpr)
+{
+    switch (wpr) {
+        case 1: return fwd_e4m3_kernel<B, NPASS, 1, STAT, GAIN, PAPER>;
+        case 2: return fwd_e4m3_kernel<B, NPASS, 2, STAT, GAIN, PAPER>;
+        case 4: return fwd_e4m3_kernel<B, NPASS, 4, STAT, GAIN, PAPER>;
+        case 8: return fwd_e4m3_kernel<B, NPASS, 8, STAT, GAIN, PAPER>;
+        case 16: return fwd_e4m3_kernel<B, NPASS, 16, STAT, GAIN, PAPER>;
+        default: break;
+    }
+    if constexpr (FINE) {
+        switch (wpr) {
+            case 3: return fwd_e4m3_kernel<B, NPASS, 3, STAT, GAIN, PAPER>;
+            case 5: return fwd_e4m3_kernel<B, NPASS, 5, STAT, GAIN, PAPER>;
+            case 6: return fwd_e4m3_kernel<B, NPASS, 6, STAT, GAIN, PAPER>;
+            case 7: return fwd_e4m3_kernel<B, NPASS, 7, STAT, GAIN, PAPER>;
+            default: break;
+        }
+    }
+    return nullptr;
+}
+
+// FINE variants exist for every pass count; the others for WPR = 1 with any pass count and for
+// WPR > 1 with the full pass count only.
 template <int B, int STAT, bool GAIN, bool PAPER>
 static fwd_fn pick_e4m3(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr == 2) return fwd_e4m3_kernel<B, MAXP, 2, STAT, GAIN, PAPER>;
-    if (wpr == 4) return fwd_e4m3_kernel<B, MAXP, 4, STAT, GAIN, PAPER>;
-    if (wpr == 8) return fwd_e4m3_kernel<B, MAXP, 8, STAT, GAIN, PAPER>;
-    if (wpr == 16) return fwd_e4m3_kernel<B, MAXP, 16, STAT, GAIN, PAPER>;
-    if (wpr != 1) return nullptr;
+    constexpr bool FINE = B == 32 && !GAIN && PAPER;
+    if (FINE || wpr > 1) {
+        if (npass == MAXP) return e4m3_by_wpr<B, MAXP, STAT, GAIN, PAPER, FINE>(wpr);
+        if (FINE && npass == 1) return e4m3_by_wpr<B, 1, STAT, GAIN, PAPER, FINE>(wpr);
+        return nullptr;
+    }
     switch (npass) {
         case 1: return fwd_e4m3_kernel<B, 1, 1, STAT, GAIN, PAPER>;
         case 2: return fwd_e4m3_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, GAIN, PAPER>;
@@ -365,33 +396,60 @@ static fwd_fn pick_round(int round, int stat, bool gain, int wpr, int npass)
 {
     return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, true>(stat, gain, wpr, npass) : pick_stat<B, false>(stat, gain, wpr, npass);
 }
+template <int NPASS>
+static fwd_fn nvfp4_by_wpr(int wpr)
+{
+    switch (wpr) {
+        case 1: return fwd_nvfp4_kernel<NPASS, 1>;
+        case 2: return fwd_nvfp4_kernel<NPASS, 2>;
+        case 3: return fwd_nvfp4_kernel<NPASS, 3>;
+        case 4: return fwd_nvfp4_kernel<NPASS, 4>;
+        case 5: return fwd_nvfp4_kernel<NPASS, 5>;
+        case 6: return fwd_nvfp4_kernel<NPASS, 6>;
+        case 7: return fwd_nvfp4_kernel<NPASS, 7>;
+        case 8: return fwd_nvfp4_kernel<NPASS, 8>;
+        case 16: return fwd_nvfp4_kernel<NPASS, 16>;
+        default: return nullptr;
+    }
+}
 static fwd_fn pick_nvfp4(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / 16;
-    if (wpr == 2) return fwd_nvfp4_kernel<MAXP, 2>;
-    if (wpr == 4) return fwd_nvfp4_kernel<MAXP, 4>;
-    if (wpr == 8) return fwd_nvfp4_kernel<MAXP, 8>;
-    if (wpr == 16) return fwd_nvfp4_kernel<MAXP, 16>;
-    if (wpr != 1) return nullptr;
-    switch (npass) {
-        case 1: return fwd_nvfp4_kernel<1, 1>;
-        case 2: return fwd_nvfp4_kernel<(MAXP >= 2 ? 2 : MAXP), 1>;
-        case 3: return fwd_nvfp4_kernel<(MAXP >= 3 ? 3 : MAXP), 1>;
-        default: return fwd_nvfp4_kernel<MAXP, 1>;
-    }
+    if (npass == MAXP) return nvfp4_by_wpr<MAXP>(wpr);
+    if (npass == MAXP / 2) return nvfp4_by_wpr<(MAXP >= 2 ? MAXP / 2 : 1)>(wpr);
+    if (npass == 1) return nvfp4_by_wpr<1>(wpr);
+    return nullptr;
 }
 
-// Splits K blocks per row over WPR warps x NPASS passes with at most MXN_FWD_MAX_ELEMS elements per lane.
-static bool plan_row(int K, int B, int* wpr, int* npass)
+// Splits the K blocks of a row over WPR warps x NPASS passes (at most MXN_FWD_MAX_ELEMS elements per
+// lane), choosing among the instantiated kernels by the fraction of idle lanes, with a handicap for
+// splits that use fewer passes than the maximum (more warps, hence more synchronisation, per row:
+// measured at D = 7168, where 4 warps x 2 passes at 87.5 % beat 7 warps x 1 pass at 100 %).
+static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
 {
     const int maxp = MXN_FWD_MAX_ELEMS / B;
-    int w = 1;
-    while ((K + 32 * w - 1) / (32 * w) > maxp) {
-        w *= 2;
-        if (w > 16) return false;
+    int best_w = 0, best_p = 0;
+    double best_cost = -1.0;
+    const int* wl = fine ? kFineWpr : kCoarseWpr;
+    const int nw = fine ? (int)(sizeof(kFineWpr) / sizeof(int)) : (int)(sizeof(kCoarseWpr) / sizeof(int));
+    for (int wi = 0; wi < nw; ++wi) {
+        const int w = wl[wi];
+        for (int p = maxp; p >= 1; --p) {
+            const bool exists = nvfp4 ? (p == maxp || p == maxp / 2 || p == 1)
+                                      : fine ? (p == maxp || p == 1) : (w == 1 || p == maxp);
+            const long lanes = (long)32 * w * p;
+            if (!exists || lanes < K) continue;
+            const double cost = (double)(lanes - K) / (double)lanes + ((p < maxp && w > 1) ? 0.15 : 0.0);
+            if (best_cost < 0.0 || cost < best_cost - 1e-9) {
+                best_cost = cost;
+                best_w = w;
+                best_p = p;
+            }
+        }
     }
-    *wpr = w;
-    *npass = (K + 32 * w - 1) / (32 * w);
+    if (best_cost < 0.0) return false;
+    *wpr = best_w;
+    *npass = best_p;
     return true;
 }
 
@@ -399,19 +457,20 @@ bool fwd_shape_supported(int64_t D, int B)
 {
     if (!(B == 16 || B == 32 || B == 64) || D <= 0 || D % B != 0 || D / B > (1 << 20)) return false;
     int wpr, npass;
-    return plan_row((int)(D / B), B, &wpr, &npass);
+    return plan_row((int)(D / B), B, false, false, &wpr, &npass);   // the coarse set is the narrowest
 }
 
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
 {
-    if (!plan_row(P.K, B, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
+    const bool fine = nvfp4 || (B == 32 && P.gain == nullptr && P.round == MXN_ROUND_RCEIL_POW2);
+    if (!plan_row(P.K, B, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
     {
         const int count = stat == STAT_RMS ? P.D : P.K;   // divisor of the row statistic
         P.inv_count = (count & (count - 1)) == 0 ? 1.0 / (double)count : 0.0;
     }
     const int warps = cta_warps(P.wpr);
-    P.rows_per_cta = warps / P.wpr;
+    P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
     if (nvfp4) fn = pick_nvfp4(P.wpr, P.npass);
     else if (B == 16) fn = pick_round<16>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);

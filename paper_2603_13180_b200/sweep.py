@@ -1,0 +1,106 @@
+"""The paper's kernel benchmark grid (appendix "Kernel Benchmarks"): tokens 2^12..2^16 x the 17 hidden
+sizes {k * 2^r, k in 1,3,5,7} within [2^10, 2^14] x block sizes, Gaussian input, forward only, norm gain
+folded away; speed-up of `mxnorm_fwd` over the fused conventional path `rmsnorm_mxfp8_fwd`, geometric mean
+over the grid.  Both sides are this library's hand-written kernels on the same GPU (the paper compares two
+torch.compile kernels on a GB200).
+
+    python -m paper_2603_13180_b200.sweep [--blocks 32] [--tokens 4096 16384 65536] [--json out.json]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+
+import torch
+
+from . import binding as mx
+
+TOKENS = [2 ** 12, 2 ** 13, 2 ** 14, 2 ** 15, 2 ** 16]
+HIDDEN = sorted({k * 2 ** r for k in (1, 3, 5, 7) for r in range(4, 15) if 2 ** 10 <= k * 2 ** r <= 2 ** 14})
+EPS = 1e-5
+
+
+def _time(fn, sets, steps, warmup, stream):
+    for i in range(warmup):
+        fn(i % sets)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for i in range(steps):
+        fn(i % sets)
+    b.record(stream)
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / steps * 1e3   # microseconds
+
+
+def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20):
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    L = mx.lib
+    rows = []
+    for B in blocks:
+        for T in tokens:
+            for D in hidden:
+                per_set = T * D * 3 + T * (D // B) + 4 * T
+                sets = max(2, min(8, -(-3 * l2_bytes // per_set)))        # working set of at least 3x L2
+                g = torch.Generator(device="cuda").manual_seed(T + D)
+                xs = [torch.randn(T, D, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(sets)]
+                outs = [mx.alloc_outputs(T, D, B, mx.SCALES_SWIZZLE_128x4) for _ in range(sets)]
+
+                def mxn(i):
+                    c, s, r = outs[i]
+                    st = L.mxnorm_fwd(xs[i].data_ptr(), None, T, D, B, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
+                                      0, mx.SCALES_SWIZZLE_128x4, sh)
+                    assert st == 0, mx.status_string(st)
+
+                def rms(i):
+                    c, s, r = outs[i]
+                    st = L.rmsnorm_mxfp8_fwd(xs[i].data_ptr(), None, T, D, B, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
+                                             0, mx.SCALES_SWIZZLE_128x4, sh)
+                    assert st == 0, mx.status_string(st)
+
+                t_mx = min(_time(mxn, sets, steps, warmup, stream) for _ in range(2))
+                t_rms = min(_time(rms, sets, steps, warmup, stream) for _ in range(2))
+                rows.append({"block": B, "tokens": T, "hidden": D, "mxnorm_us": t_mx, "rmsnorm_us": t_rms,
+                             "speedup": t_rms / t_mx, "mxnorm_gbs": per_set / t_mx / 1e3, "rmsnorm_gbs": per_set / t_rms / 1e3})
+                del xs, outs
+    return rows
+
+
+def summarise(rows):
+    out = {}
+    for B in sorted({r["block"] for r in rows}):
+        sel = [r for r in rows if r["block"] == B]
+        out[f"B={B}"] = {
+            "cases": len(sel),
+            "geomean_speedup": math.exp(sum(math.log(r["speedup"]) for r in sel) / len(sel)),
+            "max_speedup": max(r["speedup"] for r in sel),
+            "min_speedup": min(r["speedup"] for r in sel),
+            "geomean_mxnorm_gbs": math.exp(sum(math.log(r["mxnorm_gbs"]) for r in sel) / len(sel)),
+            "min_mxnorm_gbs": min(r["mxnorm_gbs"] for r in sel),
+        }
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--blocks", type=int, nargs="+", default=[32])
+    ap.add_argument("--tokens", type=int, nargs="+", default=TOKENS)
+    ap.add_argument("--hidden", type=int, nargs="+", default=HIDDEN)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--json", default="")
+    args = ap.parse_args()
+    rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps)
+    summary = summarise(rows)
+    for r in rows:
+        print(f"B={r['block']:2d} T={r['tokens']:6d} D={r['hidden']:6d}  mxnorm {r['mxnorm_us']:9.2f} us {r['mxnorm_gbs']:6.0f} GB/s   "
+              f"rmsnorm+cast {r['rmsnorm_us']:9.2f} us {r['rmsnorm_gbs']:6.0f} GB/s   speedup {r['speedup']:.3f}")
+    print(json.dumps(summary))
+    if args.json:
+        with open(args.json, "w") as f:
+            json.dump({"rows": rows, "summary": summary}, f)
+
+
+if __name__ == "__main__":
+    main()

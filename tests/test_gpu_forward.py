@@ -27,7 +27,9 @@ def rows(T, D, seed, outliers=True):
 # shapes: single lane active, ragged K (not a multiple of 32), several passes, rows spanning
 # 2/4/8 warps, odd T (ragged last CTA)
 SHAPES = [(1, 32), (5, 64), (37, 768), (130, 1024), (9, 2560), (33, 4096), (6, 5120), (5, 8192), (3, 16384),
-          (2, 32768), (257, 2048)]
+          (2, 32768), (257, 2048),
+          # hidden sizes {3,5,7} * 2^r of the paper's sweep: rows spanning 3, 5, 6 and 7 warps
+          (7, 3072), (5, 6144), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (11, 1280), (9, 1792)]
 
 
 @pytest.mark.parametrize("T,D", SHAPES)
@@ -148,7 +150,8 @@ def test_degenerate_rows(binding, oracle):
     assert np.all(scales[3] == 121) and np.all(codes[3] == 0x72) and r.view(np.uint32)[3] == 0x3ED645A2
 
 
-@pytest.mark.parametrize("T,D", [(1, 16), (5, 48), (37, 768), (130, 1024), (33, 4096), (5, 8192), (3, 16384), (257, 2048)])
+@pytest.mark.parametrize("T,D", [(1, 16), (5, 48), (37, 768), (130, 1024), (33, 4096), (5, 8192), (3, 16384), (257, 2048),
+                                 (7, 3072), (6, 5120), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (11, 1280)])
 def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
     x, _ = rows(T, D, seed=11 * T + D)
     for p, eps, gs in ((2, 1e-5, 1.0), (1, 0.0, 1.0), (2, 0.0, 8.0)):
