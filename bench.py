@@ -126,6 +126,42 @@ def time_launches(fn, n_sets: int, steps: int, warmup: int, stream) -> float:
     return start.elapsed_time(end) / steps
 
 
+def time_small_configs(mx, args, stream):
+    """Forward kernels on the small parity configs C1 [2048,768] and C2 [16384,2048] (context: C1 is
+    launch- and L2-bound, 4.8 MB in all)."""
+    out = {}
+    L, sh = mx.lib, stream.cuda_stream
+    for name in ("C1", "C2"):
+        w = wl.CONFIGS[name]
+        T, D = w.T, w.D
+        x_cpu = wl.make_inputs(w)["x"]
+        nbytes = algorithmic_bytes("mx", T, D)
+        sets = max(4, min(64, -(-3 * (126 << 20) // nbytes)))
+        xs = [x_cpu.cuda() for _ in range(sets)]
+        outs = [mx.alloc_outputs(T, D, 32, mx.SCALES_ROWMAJOR) for _ in range(sets)]
+
+        def fwd(i):
+            c, s, r = outs[i]
+            L.mxnorm_fwd(xs[i].data_ptr(), None, T, D, 32, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(), 0, 0, sh)
+
+        def rms(i):
+            c, s, r = outs[i]
+            L.rmsnorm_mxfp8_fwd(xs[i].data_ptr(), None, T, D, 32, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(), 0, 0, sh)
+
+        def cast(i):
+            c, s, r = outs[i]
+            L.mx_cast(xs[i].data_ptr(), T, D, 32, c.data_ptr(), s.data_ptr(), 0, 0, sh)
+
+        res = {}
+        for kname, fn in (("mxnorm_fwd", fwd), ("rmsnorm_mxfp8_fwd", rms), ("mx_cast", cast)):
+            ms = time_launches(fn, sets, args.steps, args.warmup, stream)
+            res[kname] = {"ms": ms, "gbs": nbytes / ms / 1e6, "tokens_per_s": T / (ms * 1e-3)}
+        res["buffer_sets"] = sets
+        out[name] = res
+        del xs, outs
+    return out
+
+
 def oracle_throughput(x_bits, reps: int = 1):
     """The CPU oracle as it stands, timed on this machine's host cores. Returns (GB/s, seconds, threads)."""
     import oracle
@@ -172,6 +208,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--skip-others", action="store_true", help="only the headline kernel (for profiler runs)")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler runs on a smaller case)")
+    ap.add_argument("--all-configs", action="store_true", help="also time the forward kernels on configs C1 and C2")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -347,6 +384,9 @@ def main():
             result["cpu_baseline"] = {"value": gbs_cpu, "unit": "GB/s", "cores": threads, "kind": "oracle",
                                       "seconds_per_batch": dt,
                                       "sample": f"20 passes of the full [{T},{D}] batch through mxnorm_ref (plain C, OpenMP over rows)"}
+
+    if args.all_configs and not args.skip_others:
+        result["configs"] = time_small_configs(mx, args, stream)
 
     if rank == 0:
         print(json.dumps(result))
