@@ -55,6 +55,11 @@ __device__ __forceinline__ float hmax_abs_to_f32(uint32_t m2)
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
+// a bf16 pair as two binary32 (exact widening) and the packed product with a broadcast factor:
+// two IEEE round-to-nearest multiplies in one instruction
+__device__ __forceinline__ float2 bf16x2_to_f32x2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+
 // ---- element casts --------------------------------------------------------------------------
 // two binary32 -> two E4M3 (RN-even, saturating to +-448); `lo` lands in the low byte
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)

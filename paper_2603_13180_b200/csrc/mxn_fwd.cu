@@ -90,7 +90,7 @@ __device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2]
 {
     constexpr int W = B / 2;
     double stat = 0.0;
-    float ss0 = 0.f, ss1 = 0.f, ss2 = 0.f, ss3 = 0.f;
+    float2 ssa = make_float2(0.f, 0.f), ssb = make_float2(0.f, 0.f);   // four binary32 partial sums of squares
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
         uint32_t m2 = absmax_bf16x2(xr[i][0], xr[i][1]);
@@ -104,16 +104,13 @@ __device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2]
         if (STAT == STAT_RMS) {
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
-                float a = bf16_lo(xr[i][j]), b = bf16_hi(xr[i][j]);
-                float c = bf16_lo(xr[i][j + 1]), d = bf16_hi(xr[i][j + 1]);
-                ss0 = __fmaf_rn(a, a, ss0);
-                ss1 = __fmaf_rn(b, b, ss1);
-                ss2 = __fmaf_rn(c, c, ss2);
-                ss3 = __fmaf_rn(d, d, ss3);
+                const float2 a = bf16x2_to_f32x2(xr[i][j]), b = bf16x2_to_f32x2(xr[i][j + 1]);
+                ssa = __ffma2_rn(a, a, ssa);
+                ssb = __ffma2_rn(b, b, ssb);
             }
         }
     }
-    if (STAT == STAT_RMS) stat = (double)ss0 + (double)ss1 + ((double)ss2 + (double)ss3);
+    if (STAT == STAT_RMS) stat = (double)ssa.x + (double)ssa.y + ((double)ssb.x + (double)ssb.y);
     return stat;
 }
 
@@ -171,17 +168,20 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
             const float f = __fmul_rn(rho, inv);
             const bool fast = sb >= 16u && rho_normal && is_normal_f32(f);
             if (__all_sync(0xFFFFFFFFu, fast || !active)) {
+                const float2 ff = make_float2(f, f);
 #pragma unroll
-                for (int j = 0; j < W; j += 2)
-                    out[j / 2] = cvt_e4m3x4(__fmul_rn(bf16_lo(xr[i][j]), f), __fmul_rn(bf16_hi(xr[i][j]), f),
-                                            __fmul_rn(bf16_lo(xr[i][j + 1]), f), __fmul_rn(bf16_hi(xr[i][j + 1]), f));
+                for (int j = 0; j < W; j += 2) {
+                    const float2 q0 = mul2(bf16x2_to_f32x2(xr[i][j]), ff), q1 = mul2(bf16x2_to_f32x2(xr[i][j + 1]), ff);
+                    out[j / 2] = cvt_e4m3x4(q0.x, q0.y, q1.x, q1.y);
+                }
             } else {
+                const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
 #pragma unroll
-                for (int j = 0; j < W; j += 2)
-                    out[j / 2] = cvt_e4m3x4(__fmul_rn(__fmul_rn(bf16_lo(xr[i][j]), rho), inv),
-                                            __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), inv),
-                                            __fmul_rn(__fmul_rn(bf16_lo(xr[i][j + 1]), rho), inv),
-                                            __fmul_rn(__fmul_rn(bf16_hi(xr[i][j + 1]), rho), inv));
+                for (int j = 0; j < W; j += 2) {
+                    const float2 q0 = mul2(mul2(bf16x2_to_f32x2(xr[i][j]), rr), ii);
+                    const float2 q1 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 1]), rr), ii);
+                    out[j / 2] = cvt_e4m3x4(q0.x, q0.y, q1.x, q1.y);
+                }
             }
         } else {
             // y = fl32(fl32(x*rho) * gamma); scales and codes from y
@@ -250,13 +250,13 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
         const float d = e4m3_to_f32(sc);
         const float inv = d == 0.0f ? 0.0f : __fdiv_rn(rho_g, d);
         uint32_t out[2];
+        const float2 ii = make_float2(inv, inv);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const uint32_t* xw = &xr[i][h * 4];
-            out[h] = cvt_e2m1x8(__fmul_rn(bf16_lo(xw[0]), inv), __fmul_rn(bf16_hi(xw[0]), inv),
-                                __fmul_rn(bf16_lo(xw[1]), inv), __fmul_rn(bf16_hi(xw[1]), inv),
-                                __fmul_rn(bf16_lo(xw[2]), inv), __fmul_rn(bf16_hi(xw[2]), inv),
-                                __fmul_rn(bf16_lo(xw[3]), inv), __fmul_rn(bf16_hi(xw[3]), inv));
+            const float2 q0 = mul2(bf16x2_to_f32x2(xw[0]), ii), q1 = mul2(bf16x2_to_f32x2(xw[1]), ii);
+            const float2 q2 = mul2(bf16x2_to_f32x2(xw[2]), ii), q3 = mul2(bf16x2_to_f32x2(xw[3]), ii);
+            out[h] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
         }
         if (k < P.K) {
             st_v2(cp0 + (int64_t)i * (WPR * kWarp * 8), out);
