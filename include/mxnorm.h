@@ -135,6 +135,21 @@ mxn_status mxnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D,
                             void* codes_u8_packed, void* scales_e4m3, float* rms_est_out_or_null,
                             mxn_scale_layout layout, void* cuda_stream);
 
+/* MXFP4 counterparts of the three forward entry points: E2M1 element values (two per byte, element 2i in
+ * the low nibble: codes_u8_packed [T, D/2], 32-byte aligned) with E8M0 block scales, B in {16, 32, 64} -
+ * the paper's cast with the element type set to E2M1 (appendix "Implementation of MXNormLinear";
+ * the kernel benchmark of Section 4.3 covers block sizes {16, 32, 64} x {E4M3, E2M1}).  The largest power
+ * of two of E2M1 is 4, so S = 2^(ceil(log2 absmax) - 2) (the paper's rounding rule; no other mode) and
+ * codes = E2M1(value / S), round-to-nearest-even, saturating at +-6.  No gain argument. */
+mxn_status mx_cast_fp4(const void* x_bf16, int64_t T, int64_t D, int block,
+                       void* codes_u8_packed, void* scales_u8, mxn_scale_layout layout, void* cuda_stream);
+mxn_status rmsnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block, float eps,
+                             void* codes_u8_packed, void* scales_u8, float* rms_out_or_null,
+                             mxn_scale_layout layout, void* cuda_stream);
+mxn_status mxnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block, int p, float coef_or_0, float eps,
+                            void* codes_u8_packed, void* scales_u8, float* rms_est_out_or_null,
+                            mxn_scale_layout layout, void* cuda_stream);
+
 /* Backward - appendix "RMSNorm gradients", used as a straight-through estimator for MXNorm
  * (Section 3.7): the RMSNorm gradient evaluated with the r the forward saved (r~ from
  * mxnorm_fwd, or the true RMS from rmsnorm_mxfp8_fwd - same formula).

@@ -21,7 +21,7 @@ OK = 0
 EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd",
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
-           "mxn_device_timeouts")
+           "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -47,11 +47,14 @@ lib.mxnorm_bwd_workspace_bytes.restype = _sz
 lib.mxnorm_fwd_host.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp, _sz, _vp]
 lib.mxnorm_fwd_host_workspace_bytes.argtypes = [_i64, _i64, _i32, _i32]
 lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
+lib.mx_cast_fp4.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
+lib.rmsnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.mxnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mxnorm_bwd_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp]
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.argtypes = []
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
 for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
-              "mxnorm_bwd_noalloc"):
+              "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd"):
     getattr(lib, _name).restype = _i32
 
 
@@ -180,3 +183,24 @@ def mxnorm_bwd_noalloc(x, grad_out, gain, rms, dx, dgain=None, stream=None):
     _check(lib.mxnorm_bwd_noalloc(_ptr(x), _ptr(grad_out), _ptr(gain), _ptr(rms), T, D, _ptr(dx),
                                   1 if dx.dtype == torch.float32 else 0, _ptr(dgain), _stream(stream)),
            "mxnorm_bwd_noalloc")
+
+
+def mx_cast_fp4(x, codes_packed, scales, block=32, layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mx_cast_fp4(_ptr(x), T, D, block, _ptr(codes_packed), _ptr(scales), layout, _stream(stream)), "mx_cast_fp4")
+
+
+def rmsnorm_mxfp4_fwd(x, codes_packed, scales, rms_out=None, eps=0.0, block=32, layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.rmsnorm_mxfp4_fwd(_ptr(x), T, D, block, eps, _ptr(codes_packed), _ptr(scales), _ptr(rms_out), layout,
+                                 _stream(stream)), "rmsnorm_mxfp4_fwd")
+
+
+def mxnorm_mxfp4_fwd(x, codes_packed, scales, rms_est_out=None, p=2, coef=0.0, eps=0.0, block=32,
+                     layout=SCALES_ROWMAJOR, stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mxnorm_mxfp4_fwd(_ptr(x), T, D, block, p, coef, eps, _ptr(codes_packed), _ptr(scales), _ptr(rms_est_out),
+                                layout, _stream(stream)), "mxnorm_mxfp4_fwd")

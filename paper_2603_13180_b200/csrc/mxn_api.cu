@@ -44,7 +44,7 @@ cudaError_t clear_scale_padding(void* scales, int64_t T, int64_t K, int layout, 
 
 mxn_status run_fwd(int stat, bool nvfp4, const void* x, const void* gain, int64_t T, int64_t D, int B, int p,
                    float coef, float eps, float global_scale, void* codes, void* scales, float* rms,
-                   int round, int layout, void* stream)
+                   int round, int layout, void* stream, int elem = mxn::ELEM_E4M3)
 {
     mxn_status st = check_common(x, T, D, B, codes, scales, round, layout);
     if (st != MXN_OK || T == 0) return st;
@@ -70,6 +70,7 @@ mxn_status run_fwd(int stat, bool nvfp4, const void* x, const void* gain, int64_
     P.global_scale = global_scale;
     P.round = round;
     P.layout = layout;
+    P.elem = nvfp4 ? mxn::ELEM_E2M1 : elem;
     if (clear_scale_padding(scales, T, P.K, layout, s) != cudaSuccess) return MXN_ERR_CUDA;
     return mxn::launch_fwd(P, B, stat, nvfp4, s) == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
 }
@@ -142,6 +143,28 @@ mxn_status mxnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int p, flo
 {
     return run_fwd(mxn::STAT_MX, true, x_bf16, nullptr, T, D, 16, p, coef_or_0, eps, global_scale, codes_u8_packed,
                    scales_e4m3, rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
+}
+
+mxn_status mx_cast_fp4(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8_packed, void* scales_u8,
+                       mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_fwd(mxn::STAT_NONE, false, x_bf16, nullptr, T, D, block, 2, 1.0f, 0.0f, 1.0f, codes_u8_packed, scales_u8,
+                   nullptr, MXN_ROUND_RCEIL_POW2, layout, cuda_stream, mxn::ELEM_E2M1);
+}
+
+mxn_status rmsnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block, float eps, void* codes_u8_packed,
+                             void* scales_u8, float* rms_out_or_null, mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_fwd(mxn::STAT_RMS, false, x_bf16, nullptr, T, D, block, 2, 1.0f, eps, 1.0f, codes_u8_packed, scales_u8,
+                   rms_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream, mxn::ELEM_E2M1);
+}
+
+mxn_status mxnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block, int p, float coef_or_0, float eps,
+                            void* codes_u8_packed, void* scales_u8, float* rms_est_out_or_null,
+                            mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_fwd(mxn::STAT_MX, false, x_bf16, nullptr, T, D, block, p, coef_or_0, eps, 1.0f, codes_u8_packed, scales_u8,
+                   rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream, mxn::ELEM_E2M1);
 }
 
 mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,

@@ -230,6 +230,58 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
     }
 }
 
+// phase 2 (MXFP4: E2M1 codes two per byte, E8M0 scales; the paper's rounding rule with 4 = 2^2 as the
+// largest power of two of the element format): S = 2^(ceil(log2 a) - 2)
+template <int B, int NPASS, int WPR>
+__device__ __forceinline__ void quantise_store_mxfp4(const uint32_t (&xr)[NPASS][B / 2], const float (&m)[NPASS], float rho,
+                                                     const FwdParams& P, int64_t row, int w, int lane)
+{
+    constexpr int W = B / 2;
+    const bool rho_normal = is_normal_f32(rho);
+    uint8_t* cp0 = P.codes + row * (P.D / 2) + (int64_t)(w * kWarp + lane) * (B / 2);
+    int64_t soff, sstep;
+    scale_addressing<WPR>(P, row, w, lane, soff, sstep);
+    uint8_t* sp0 = P.scales + soff;
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        const int k = (i * WPR + w) * kWarp + lane;
+        const bool active = k < P.K;
+        const float a = __fmul_rn(m[i], rho);
+        const uint32_t u = __float_as_uint(a), E = u >> 23;
+        uint32_t sb;
+        if (E >= 255u) sb = (u & 0x7FFFFFu) ? 0u : 254u;   // not finite (outside the contract)
+        else sb = (uint32_t)max((int)E + ((u & 0x7FFFFFu) != 0u) - 2, 0);
+        const float inv = inv_scale(sb);
+        const float f = __fmul_rn(rho, inv);
+        const bool fast = sb >= 16u && rho_normal && is_normal_f32(f);   // same argument as for E4M3
+        uint32_t out[W / 4];
+        if (__all_sync(0xFFFFFFFFu, fast || !active)) {
+            const float2 ff = make_float2(f, f);
+#pragma unroll
+            for (int j = 0; j < W; j += 4) {
+                const float2 q0 = mul2(bf16x2_to_f32x2(xr[i][j]), ff), q1 = mul2(bf16x2_to_f32x2(xr[i][j + 1]), ff);
+                const float2 q2 = mul2(bf16x2_to_f32x2(xr[i][j + 2]), ff), q3 = mul2(bf16x2_to_f32x2(xr[i][j + 3]), ff);
+                out[j / 4] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
+            }
+        } else {
+            const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
+#pragma unroll
+            for (int j = 0; j < W; j += 4) {
+                const float2 q0 = mul2(mul2(bf16x2_to_f32x2(xr[i][j]), rr), ii), q1 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 1]), rr), ii);
+                const float2 q2 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 2]), rr), ii), q3 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 3]), rr), ii);
+                out[j / 4] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
+            }
+        }
+        if (active) {
+            uint8_t* cp = cp0 + (int64_t)i * (WPR * kWarp * (B / 2));
+            if (B == 16) st_v2(cp, out);
+            else if (B == 32) st_v4(cp, out);
+            else st_v8(cp, out);
+            sp0[i * sstep] = (uint8_t)sb;
+        }
+    }
+}
+
 // phase 2 (NVFP4): E4M3 block scales, E2M1 codes two per byte, B = 16
 template <int NPASS, int WPR>
 __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS][8], const float (&m)[NPASS], float rho,
@@ -307,6 +359,31 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m
         if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     }
     quantise_store_e4m3<B, NPASS, WPR, GAIN, PAPER>(xr, m, rho, P, row, w, lane);
+}
+
+// E2M1 codes with E8M0 scales (MXFP4): no gain, the paper's rounding rule
+template <int B, int NPASS, int WPR, int STAT>
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxfp4_kernel(const FwdParams P)
+{
+    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / WPR, w = warp - group * WPR;
+    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    pdl_prologue();
+    if (row >= P.T) return;
+
+    uint32_t xr[NPASS][B / 2];
+    float m[NPASS];
+    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
+    double stat = block_stats<B, NPASS, STAT>(xr, m, P.p);
+    if (STAT == STAT_RMS) forget_unpacked<NPASS, B / 2>(xr);
+    float r = 1.0f, rho = 1.0f;
+    if (STAT != STAT_NONE) {
+        stat = group_sum<WPR>(stat, group, w, red);
+        finish_stat<STAT>(stat, P, r, rho);
+        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    }
+    quantise_store_mxfp4<B, NPASS, WPR>(xr, m, rho, P, row, w, lane);
 }
 
 template <int NPASS, int WPR>
@@ -396,6 +473,30 @@ static fwd_fn pick_round(int round, int stat, bool gain, int wpr, int npass)
 {
     return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, true>(stat, gain, wpr, npass) : pick_stat<B, false>(stat, gain, wpr, npass);
 }
+template <int B, int STAT>
+static fwd_fn pick_mxfp4(int wpr, int npass)
+{
+    constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
+    if (wpr == 2) return fwd_mxfp4_kernel<B, MAXP, 2, STAT>;
+    if (wpr == 4) return fwd_mxfp4_kernel<B, MAXP, 4, STAT>;
+    if (wpr == 8) return fwd_mxfp4_kernel<B, MAXP, 8, STAT>;
+    if (wpr == 16) return fwd_mxfp4_kernel<B, MAXP, 16, STAT>;
+    if (wpr != 1) return nullptr;
+    switch (npass) {
+        case 1: return fwd_mxfp4_kernel<B, 1, 1, STAT>;
+        case 2: return fwd_mxfp4_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT>;
+        case 3: return fwd_mxfp4_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT>;
+        default: return fwd_mxfp4_kernel<B, MAXP, 1, STAT>;
+    }
+}
+template <int B>
+static fwd_fn pick_mxfp4_stat(int stat, int wpr, int npass)
+{
+    if (stat == STAT_MX) return pick_mxfp4<B, STAT_MX>(wpr, npass);
+    if (stat == STAT_RMS) return pick_mxfp4<B, STAT_RMS>(wpr, npass);
+    return pick_mxfp4<B, STAT_NONE>(wpr, npass);
+}
+
 template <int NPASS>
 static fwd_fn nvfp4_by_wpr(int wpr)
 {
@@ -462,7 +563,8 @@ bool fwd_shape_supported(int64_t D, int B)
 
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
 {
-    const bool fine = nvfp4 || (B == 32 && P.gain == nullptr && P.round == MXN_ROUND_RCEIL_POW2);
+    const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
+    const bool fine = nvfp4 || (!mxfp4 && B == 32 && P.gain == nullptr && P.round == MXN_ROUND_RCEIL_POW2);
     if (!plan_row(P.K, B, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
     {
@@ -473,6 +575,8 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
     if (nvfp4) fn = pick_nvfp4(P.wpr, P.npass);
+    else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16>(stat, P.wpr, P.npass)
+                       : B == 32 ? pick_mxfp4_stat<32>(stat, P.wpr, P.npass) : pick_mxfp4_stat<64>(stat, P.wpr, P.npass);
     else if (B == 16) fn = pick_round<16>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
     else if (B == 32) fn = pick_round<32>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
     else fn = pick_round<64>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);

@@ -7,6 +7,7 @@
 namespace mxn {
 
 enum { STAT_NONE = 0, STAT_RMS = 1, STAT_MX = 2 };
+enum { ELEM_E4M3 = 0, ELEM_E2M1 = 1 };
 
 struct FwdParams {
     const uint16_t* x;      // bf16 [T, D]
@@ -19,6 +20,7 @@ struct FwdParams {
     int p;
     float coef, eps, global_scale;
     int round, layout;
+    int elem;               // ELEM_E4M3 (one byte per element) or ELEM_E2M1 (two elements per byte)
     // filled by the launcher
     int wpr, npass, rows_per_cta, tiles_per_row;
     double inv_count;       // 1/K (MXNorm) or 1/D (RMSNorm) when that is a power of two (exact), else 0

@@ -4,7 +4,7 @@ folded away; speed-up of `mxnorm_fwd` over the fused conventional path `rmsnorm_
 over the grid.  Both sides are this library's hand-written kernels on the same GPU (the paper compares two
 torch.compile kernels on a GB200).
 
-    python -m paper_2603_13180_b200.sweep [--blocks 32] [--tokens 4096 16384 65536] [--json out.json]
+    python -m paper_2603_13180_b200.sweep [--blocks 32] [--elem e4m3|e2m1] [--tokens 4096 16384 65536] [--json out.json]
 """
 from __future__ import annotations
 
@@ -34,7 +34,7 @@ def _time(fn, sets, steps, warmup, stream):
     return a.elapsed_time(b) / steps * 1e3   # microseconds
 
 
-def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20):
+def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4m3"):
     stream = torch.cuda.current_stream()
     sh = stream.cuda_stream
     L = mx.lib
@@ -42,27 +42,38 @@ def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20):
     for B in blocks:
         for T in tokens:
             for D in hidden:
-                per_set = T * D * 3 + T * (D // B) + 4 * T
+                fp4 = elem == "e2m1"
+                per_set = T * D * 2 + (T * D // 2 if fp4 else T * D) + T * (D // B) + 4 * T
                 sets = max(2, min(8, -(-3 * l2_bytes // per_set)))        # working set of at least 3x L2
                 g = torch.Generator(device="cuda").manual_seed(T + D)
                 xs = [torch.randn(T, D, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(sets)]
-                outs = [mx.alloc_outputs(T, D, B, mx.SCALES_SWIZZLE_128x4) for _ in range(sets)]
+                outs = [mx.alloc_outputs(T, D, B, mx.SCALES_SWIZZLE_128x4, nvfp4=fp4) for _ in range(sets)]
 
                 def mxn(i):
                     c, s, r = outs[i]
+                    if fp4:
+                        st = L.mxnorm_mxfp4_fwd(xs[i].data_ptr(), T, D, B, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
+                                                mx.SCALES_SWIZZLE_128x4, sh)
+                        assert st == 0, mx.status_string(st)
+                        return
                     st = L.mxnorm_fwd(xs[i].data_ptr(), None, T, D, B, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
                                       0, mx.SCALES_SWIZZLE_128x4, sh)
                     assert st == 0, mx.status_string(st)
 
                 def rms(i):
                     c, s, r = outs[i]
+                    if fp4:
+                        st = L.rmsnorm_mxfp4_fwd(xs[i].data_ptr(), T, D, B, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
+                                                 mx.SCALES_SWIZZLE_128x4, sh)
+                        assert st == 0, mx.status_string(st)
+                        return
                     st = L.rmsnorm_mxfp8_fwd(xs[i].data_ptr(), None, T, D, B, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
                                              0, mx.SCALES_SWIZZLE_128x4, sh)
                     assert st == 0, mx.status_string(st)
 
                 t_mx = min(_time(mxn, sets, steps, warmup, stream) for _ in range(2))
                 t_rms = min(_time(rms, sets, steps, warmup, stream) for _ in range(2))
-                rows.append({"block": B, "tokens": T, "hidden": D, "mxnorm_us": t_mx, "rmsnorm_us": t_rms,
+                rows.append({"elem": elem, "block": B, "tokens": T, "hidden": D, "mxnorm_us": t_mx, "rmsnorm_us": t_rms,
                              "speedup": t_rms / t_mx, "mxnorm_gbs": per_set / t_mx / 1e3, "rmsnorm_gbs": per_set / t_rms / 1e3})
                 del xs, outs
     return rows
@@ -89,12 +100,13 @@ def main():
     ap.add_argument("--tokens", type=int, nargs="+", default=TOKENS)
     ap.add_argument("--hidden", type=int, nargs="+", default=HIDDEN)
     ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--elem", default="e4m3", choices=["e4m3", "e2m1"], help="element format (E8M0 scales either way)")
     ap.add_argument("--json", default="")
     args = ap.parse_args()
-    rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps)
+    rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps, elem=args.elem)
     summary = summarise(rows)
     for r in rows:
-        print(f"B={r['block']:2d} T={r['tokens']:6d} D={r['hidden']:6d}  mxnorm {r['mxnorm_us']:9.2f} us {r['mxnorm_gbs']:6.0f} GB/s   "
+        print(f"{r['elem']} B={r['block']:2d} T={r['tokens']:6d} D={r['hidden']:6d}  mxnorm {r['mxnorm_us']:9.2f} us {r['mxnorm_gbs']:6.0f} GB/s   "
               f"rmsnorm+cast {r['rmsnorm_us']:9.2f} us {r['rmsnorm_gbs']:6.0f} GB/s   speedup {r['speedup']:.3f}")
     print(json.dumps(summary))
     if args.json:

@@ -37,9 +37,10 @@ def run_fwd(binding, oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coe
     x = wl.from_bits(x_bits).cuda()
     gain = None if gain_bits is None else wl.from_bits(gain_bits).cuda()
     nvfp4 = kind == "nvfp4"
+    fp4 = nvfp4 or kind in ("cast4", "rms4", "mx4")     # E2M1 codes: two elements per byte
     B = 16 if nvfp4 else block
     K = D // B
-    ccols = D // 2 if nvfp4 else D
+    ccols = D // 2 if fp4 else D
     cfull, codes = guarded(T * ccols)
     sbytes = binding.scale_bytes(T, K, layout)
     sfull, scales = guarded(sbytes)
@@ -57,6 +58,13 @@ def run_fwd(binding, oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coe
     elif kind == "nvfp4":
         binding.mxnorm_nvfp4_fwd(x, codes, scales, rms, p=p, coef=coef, eps=eps, global_scale=global_scale,
                                  layout=layout)
+    elif kind == "cast4":
+        binding.mx_cast_fp4(x, codes, scales, block=B, layout=layout)
+        rms = None
+    elif kind == "rms4":
+        binding.rmsnorm_mxfp4_fwd(x, codes, scales, rms, eps=eps, block=B, layout=layout)
+    elif kind == "mx4":
+        binding.mxnorm_mxfp4_fwd(x, codes, scales, rms, p=p, coef=coef, eps=eps, block=B, layout=layout)
     else:
         raise ValueError(kind)
     torch.cuda.synchronize()
@@ -83,6 +91,13 @@ def run_ref(oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coef=0.0, ep
         return oracle.mxnorm_ref(x_bits, gain=gain_bits, p=p, coef=coef, eps=eps, block=block, mode=round)
     if kind == "nvfp4":
         return oracle.mxnorm_nvfp4_ref(x_bits, p=p, coef=coef, eps=eps, global_scale=global_scale)
+    if kind == "cast4":
+        c, s = oracle.mx_cast_ref(x_bits, block=block, elem=oracle.ELEM_E2M1)
+        return c, s, None
+    if kind == "rms4":
+        return oracle.rmsnorm_mxfp8_ref(x_bits, eps=eps, block=block, elem=oracle.ELEM_E2M1)
+    if kind == "mx4":
+        return oracle.mxnorm_ref(x_bits, p=p, coef=coef, eps=eps, block=block, elem=oracle.ELEM_E2M1)
     raise ValueError(kind)
 
 
@@ -101,7 +116,17 @@ def assert_exact(got, want, what=""):
         assert np.array_equal(gr.view(np.uint32), wr.view(np.uint32)), f"{what}: rms differs"
 
 
-def assert_within_rounding_of_rho(got, want, block, what=""):
+def nibble_steps(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """per-element code-step distance of packed E2M1 bytes (two sign-magnitude nibbles per byte)"""
+    def sm(n):
+        mag = (n & 7).astype(np.int32)
+        return np.where(n & 8, -mag, mag)
+    lo = np.abs(sm(a & 0xF) - sm(b & 0xF))
+    hi = np.abs(sm(a >> 4) - sm(b >> 4))
+    return np.stack([lo, hi], axis=-1).reshape(a.shape[0], -1)
+
+
+def assert_within_rounding_of_rho(got, want, block, what="", fp4=False):
     """Tolerance for a path whose fp32 normalisation factor may round differently from the oracle's
     (the binary32 sum of squares of the RMSNorm baseline): r within 1e-6 relative; scale bytes may
     differ (by one) in at most 1e-6 of the blocks; outside those blocks at most 1e-4 of the codes
@@ -113,7 +138,7 @@ def assert_within_rounding_of_rho(got, want, block, what=""):
     assert sdiff.mean() <= 1e-6 or sdiff.sum() <= 1, f"{what}: {sdiff.sum()} scales differ"
     assert np.all(np.abs(gs.astype(int) - ws.astype(int)) <= 1)
     keep = ~np.repeat(sdiff, block, axis=1)
-    d = np.abs(sm_int(gc) - sm_int(wc))[keep]
+    d = (nibble_steps(gc, wc) if fp4 else np.abs(sm_int(gc) - sm_int(wc)))[keep]
     assert d.max(initial=0) <= 1, f"{what}: a code differs by more than one step"
     assert (d != 0).mean() <= 1e-4, f"{what}: {(d != 0).mean():.2e} of codes differ"
     return int(sdiff.sum()), int((d != 0).sum())

@@ -65,6 +65,10 @@ def test_argument_errors_are_statuses(binding):
     assert L.rmsnorm_mxfp8_fwd(FAKE, FAKE + 2, 4, 128, 32, 0.0, FAKE, FAKE, None, 0, 0, None) == 3
     assert L.mxnorm_nvfp4_fwd(FAKE, 4, 100, 2, 0.0, 0.0, 1.0, FAKE, FAKE, None, 0, None) == 2
     assert L.mxnorm_nvfp4_fwd(FAKE, 0, 128, 2, 0.0, 0.0, 1.0, FAKE, FAKE, None, 0, None) == 0
+    assert L.mxnorm_mxfp4_fwd(FAKE, 4, 100, 32, 2, 0.0, 0.0, FAKE, FAKE, None, 0, None) == 2
+    assert L.mxnorm_mxfp4_fwd(FAKE, 4, 128, 32, 5, 0.0, 0.0, FAKE, FAKE, None, 0, None) == 2
+    assert L.mx_cast_fp4(FAKE, 4, 128, 32, None, FAKE, 0, None) == 1
+    assert L.rmsnorm_mxfp4_fwd(FAKE, 4, 128, 32, 0.0, FAKE, FAKE, None, 3, None) == 4
     # backward
     ws = binding.mxnorm_bwd_workspace_bytes(64, 4096)
     assert ws > 0 and ws % (4096 * 4) == 0

@@ -190,3 +190,36 @@ def test_rms_output_is_optional_and_stream_is_honoured(binding, oracle):
     s.synchronize()
     want = gu.run_ref(oracle, "mx", x_bits, eps=1e-5)
     assert np.array_equal(codes.cpu().numpy(), want[0]) and np.array_equal(scales.cpu().numpy().reshape(64, 32), want[1])
+
+
+@pytest.mark.parametrize("block", [16, 32, 64])
+@pytest.mark.parametrize("T,D", [(1, 64), (37, 768), (130, 1024), (33, 4096), (9, 2560), (5, 8192), (3, 16384), (257, 2048)])
+def test_mxfp4_matches_oracle(binding, oracle, T, D, block):
+    """E2M1 codes with E8M0 scales (the paper's cast with the element type set to E2M1)."""
+    x, _ = rows(T, D, seed=13 * T + D + block)
+    for p, eps in ((2, 1e-5), (1, 0.0)):
+        got = gu.run_fwd(binding, oracle, "mx4", x, block=block, p=p, eps=eps)
+        gu.assert_exact(got, gu.run_ref(oracle, "mx4", x, block=block, p=p, eps=eps), f"mxnorm_mxfp4 B={block} p={p} {T}x{D}")
+    got = gu.run_fwd(binding, oracle, "cast4", x, block=block)
+    gu.assert_exact(got, gu.run_ref(oracle, "cast4", x, block=block), f"mx_cast_fp4 B={block}")
+    got = gu.run_fwd(binding, oracle, "rms4", x, block=block, eps=1e-5)
+    gu.assert_within_rounding_of_rho(got, gu.run_ref(oracle, "rms4", x, block=block, eps=1e-5), block, "rmsnorm_mxfp4", fp4=True)
+    got = gu.run_fwd(binding, oracle, "mx4", x, block=block, eps=1e-5, layout=1)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx4", x, block=block, eps=1e-5), "mxnorm_mxfp4 tiled scales")
+
+
+def test_mxfp4_degenerate_rows_and_patterns(binding, oracle):
+    pats = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    pats = pats[(pats & 0x7F80) != 0x7F80]
+    x = np.zeros((pats.size, 32), np.uint16)
+    x[:, 0] = pats
+    x[:, 17] = (pats >> 1) & 0x7FFF
+    x[(x[:, 17] & 0x7F80) == 0x7F80, 17] = 0
+    gu.assert_exact(gu.run_fwd(binding, oracle, "cast4", x), gu.run_ref(oracle, "cast4", x), "fp4 patterns")
+    z = np.zeros((4, 128), np.uint16)
+    z[1, :] = 0x8000
+    z[2, 7] = 0x3F80
+    z[3, :] = 0x3F80
+    codes, scales, r = gu.run_fwd(binding, oracle, "mx4", z)
+    gu.assert_exact((codes, scales, r), gu.run_ref(oracle, "mx4", z), "fp4 degenerate")
+    assert np.all(scales[3] == 127) and np.all(codes[3] == 0x44)      # constant row closed form

@@ -340,6 +340,53 @@ def test_nvfp4_scales_and_codes_by_definition_given_rho(oracle):
         assert np.all(np.abs(deq - ynorm) <= 0.25 * np.repeat(a, 16, axis=1) + 1e-6)
 
 
+def test_mxfp4_element_format_by_definition(oracle):
+    """E2M1 values with E8M0 scales (the listing's cast with dtype = E2M1): the largest power of two of the
+    format is 4, so S is the smallest power of two with absmax/S <= 4; codes are the nearest E2M1 values,
+    two per byte (element 2i in the low nibble)."""
+    E2 = oracle.ELEM_E2M1
+    x = wl.bits(wl.make_inputs(wl.Workload("t", 20, 512, seed=12, outlier_frac=0.004))["x"])
+    xv = bf16_vals(x)
+
+    def check(codes, scales, y, B):
+        m = np.abs(y).reshape(y.shape[0], -1, B).max(-1)
+        sb = smallest_pow2_scale(m, emax=2)
+        assert np.array_equal(scales, sb)
+        S = np.repeat(np.ldexp(1.0, sb.astype(int) - 127), B, axis=1)
+        code, neg = nearest_code(y.astype(np.float64) / S, E2M1_POS)
+        nib = code | (neg.astype(np.uint8) << 3)
+        assert np.array_equal(codes, nib[:, 0::2] | (nib[:, 1::2] << 4))
+
+    for B in (16, 32, 64):
+        codes, scales = oracle.mx_cast_ref(x, block=B, elem=E2)
+        check(codes, scales, xv, B)
+        codes, scales, r = oracle.mxnorm_ref(x, eps=1e-5, block=B, elem=E2)
+        rho = (np.float32(1.0) / (r + np.float32(1e-5))).astype(np.float32)
+        check(codes, scales, (xv * rho[:, None]).astype(np.float32), B)
+        # the estimate does not depend on the element format
+        assert np.array_equal(r, oracle.mxnorm_ref(x, eps=1e-5, block=B)[2])
+        codes, scales, r = oracle.rmsnorm_mxfp8_ref(x, eps=1e-5, block=B, elem=E2)
+        rho = (np.float32(1.0) / r).astype(np.float32)
+        check(codes, scales, (xv * rho[:, None]).astype(np.float32), B)
+    # constant row: x*rho~ = 2.389 in (2,4] -> S = 1 (biased 127), nearest E2M1 value 2 -> nibble 4 -> byte 0x44
+    ones = np.full((2, 64), ONE, np.uint16)
+    codes, scales, _ = oracle.mxnorm_ref(ones, elem=E2)
+    assert np.all(scales == 127) and np.all(codes == 0x44)
+    # 2^k shifts and all bf16 patterns as lone block maxima
+    xs = bf16_bits(xv * np.float32(2.0 ** 5))
+    c0, s0 = oracle.mx_cast_ref(x, elem=E2)
+    c1, s1 = oracle.mx_cast_ref(xs, elem=E2)
+    assert np.array_equal(c0, c1) and np.array_equal(s1.astype(int), s0.astype(int) + 5)
+    pats = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    pats = pats[(pats & 0x7F80) != 0x7F80]
+    xp = np.zeros((pats.size, 32), np.uint16)
+    xp[:, 0] = pats
+    xp[:, 1] = (pats >> 1) & 0x7FFF
+    xp[(xp[:, 1] & 0x7F80) == 0x7F80, 1] = 0
+    codes, scales = oracle.mx_cast_ref(xp, elem=E2)
+    check(codes, scales, bf16_vals(xp), 32)
+
+
 # ------------------------------------------------------------------ library restatements
 def test_rms_estimate_against_numpy_restatement(oracle):
     x = _rand_rows(7, T=64, D=1024)
