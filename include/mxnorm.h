@@ -150,6 +150,18 @@ mxn_status mxnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block,
                             void* codes_u8_packed, void* scales_u8, float* rms_est_out_or_null,
                             mxn_scale_layout layout, void* cuda_stream);
 
+/* Column-wise (transposed) MXCast for the weight-gradient GEMM of MXNormLinear - Section 3.7,
+ * grad W = MXCast(grad H^T) MXCast(rho~ X) gamma: the forward's MX tensor is block-quantised along the hidden
+ * axis and cannot be reused, so the activation is re-quantised along the TOKEN axis from the cached X and r~.
+ *   y_td = x_td * rho_t with rho_t = 1 / (rms_or_null[t] + eps) (0 when the denominator is 0), or y = x when
+ *   rms_or_null is NULL (e.g. for the upstream gradient).  Blocks are 32 consecutive tokens of one column;
+ *   S and codes as in mx_cast.  Outputs are laid out transposed: codes_t_u8 [D, T] (32-byte aligned),
+ *   scales_t_u8 [D, T/32] row-major or tiled with D as the row index (mxn_scale_bytes(D, T/32, layout)).
+ *   Requires T % 32 == 0 and D % 4 == 0; x 8-byte aligned. */
+mxn_status mx_cast_transposed(const void* x_bf16, const float* rms_or_null, int64_t T, int64_t D, float eps,
+                              void* codes_t_u8, void* scales_t_u8,
+                              mxn_round round, mxn_scale_layout layout, void* cuda_stream);
+
 /* Backward - appendix "RMSNorm gradients", used as a straight-through estimator for MXNorm
  * (Section 3.7): the RMSNorm gradient evaluated with the r the forward saved (r~ from
  * mxnorm_fwd, or the true RMS from rmsnorm_mxfp8_fwd - same formula).

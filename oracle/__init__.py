@@ -50,6 +50,8 @@ def _load():
         lib.mxnorm_ref.argtypes = [vp, vp, i64, i64, i32, i32, f32, f32, i32, i32, vp, vp, vp]
         lib.mxnorm_nvfp4_ref.argtypes = [vp, i64, i64, i32, f32, f32, f32, vp, vp, vp]
         lib.mxnorm_bwd_ref.argtypes = [vp, vp, vp, vp, i64, i64, vp, vp]
+        lib.mx_cast_transposed_ref.argtypes = [vp, vp, i64, i64, i32, f32, i32, vp, vp]
+        lib.mx_cast_transposed_ref.restype = i32
         for f in (lib.mx_cast_ref, lib.rmsnorm_mxfp8_ref, lib.mxnorm_ref, lib.mxnorm_nvfp4_ref,
                   lib.mxnorm_bwd_ref):
             f.restype = i32
@@ -164,6 +166,18 @@ def mxnorm_bwd_ref(x, g, gain, rms, want_dx=True, want_dgain=True):
     _check(_load().mxnorm_bwd_ref(_p(x), _p(g), _p(gn), _p(rms), T, D, _p(dx), _p(dg)),
            "mxnorm_bwd_ref")
     return dx, dg
+
+
+def mx_cast_transposed_ref(x, rms=None, eps=0.0, block=32, mode=ROUND_RCEIL_POW2):
+    """Column-wise MXCast of x * rho (rho = 1/(rms+eps), or 1): returns (codes [D, T] u8, scales [D, T/block] u8)."""
+    x = _bf16(x, 2)
+    T, D = x.shape
+    r = None if rms is None else np.ascontiguousarray(rms, dtype=np.float32)
+    codes = np.zeros((D, T), np.uint8)
+    scales = np.zeros((D, T // block if T % block == 0 else 0), np.uint8)
+    _check(_load().mx_cast_transposed_ref(_p(x), _p(r), T, D, block, eps, mode, _p(codes), _p(scales)),
+           "mx_cast_transposed_ref")
+    return codes, scales
 
 
 def swizzle_offset(r: int, c: int, K: int) -> int:

@@ -18,7 +18,7 @@
  * [reading]; the project's design document lists them all.
  *
  * Pin status (see tests/test_oracle_*.py):
- *   mx_cast_ref, rmsnorm_mxfp8_ref, mxnorm_ref, mxnorm_bwd_ref : pinned
+ *   mx_cast_ref, rmsnorm_mxfp8_ref, mxnorm_ref, mxnorm_bwd_ref, mx_cast_transposed_ref : pinned
  *     (printed constants and bounds, closed forms, invariants, brute force,
  *      library special cases, finite differences).
  *   mxnorm_nvfp4_ref : PARITY UNPINNED by the paper - the paper gives only
@@ -427,6 +427,45 @@ int mxnorm_bwd_ref(const uint16_t *x_bf16, const uint16_t *g_bf16, const uint16_
             double h = g * gam;
             if (dx) dx[t * D + d] = h / r - x * delta / (r * r * r);
             if (dgain) dgain[d] += (x / r) * g;
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* O6  Column-wise (transposed) MXCast for the weight-gradient GEMM            */
+/*     (Section "MXNormLinear": grad W = MXCast(grad H^T) MXCast(rho~ X) gamma,*/
+/*     where the activation must be block-quantised along the TOKEN axis).     */
+/*     y_td = fl32(x_td * rho_t), rho_t = fl32(1 / fl32(r_t + eps)) (0 when    */
+/*     the denominator is 0) or 1 when no r is given; blocks are B consecutive */
+/*     tokens of one column; S, V as in MXCast; outputs are laid out           */
+/*     transposed: codes [D, T], scales [D, T/B].                              */
+/* ------------------------------------------------------------------------- */
+int mx_cast_transposed_ref(const uint16_t *x_bf16, const float *rms_or_null, int64_t T, int64_t D, int B,
+                           float eps, int mode, uint8_t *codes_t, uint8_t *scales_t)
+{
+    if (T < 0 || D <= 0 || !(B == 16 || B == 32 || B == 64) || T % B != 0) return 1;
+    int64_t KT = T / B;
+#pragma omp parallel for schedule(static)
+    for (int64_t d = 0; d < D; ++d) {
+        for (int64_t k = 0; k < KT; ++k) {
+            float y[64];
+            float m = 0.0f;
+            for (int b = 0; b < B; ++b) {
+                int64_t t = k * B + b;
+                float rho = 1.0f;
+                if (rms_or_null) {
+                    float den = rms_or_null[t] + eps;
+                    rho = den == 0.0f ? 0.0f : 1.0f / den;
+                }
+                y[b] = bf16_to_f32(x_bf16[t * D + d]) * rho;
+                float a = fabsf(y[b]);
+                if (a > m) m = a;
+            }
+            uint8_t sb = e8m0_scale(m, mode, REF_ELEM_E4M3);
+            scales_t[d * KT + k] = sb;
+            float inv = inv_scale_f32(sb);
+            for (int b = 0; b < B; ++b) codes_t[d * T + k * B + b] = e4m3_encode(y[b] * inv);
         }
     }
     return 0;

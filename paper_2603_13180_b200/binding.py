@@ -21,7 +21,8 @@ OK = 0
 EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd",
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
-           "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd")
+           "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
+           "mx_cast_transposed")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -50,11 +51,13 @@ lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
 lib.mx_cast_fp4.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.rmsnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mxnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.mx_cast_transposed.argtypes = [_vp, _vp, _i64, _i64, _f32, _vp, _vp, _i32, _i32, _vp]
 lib.mxnorm_bwd_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp]
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.argtypes = []
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
 for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
-              "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd"):
+              "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
+           "mx_cast_transposed"):
     getattr(lib, _name).restype = _i32
 
 
@@ -204,3 +207,11 @@ def mxnorm_mxfp4_fwd(x, codes_packed, scales, rms_est_out=None, p=2, coef=0.0, e
     T, D = x.shape
     _check(lib.mxnorm_mxfp4_fwd(_ptr(x), T, D, block, p, coef, eps, _ptr(codes_packed), _ptr(scales), _ptr(rms_est_out),
                                 layout, _stream(stream)), "mxnorm_mxfp4_fwd")
+
+
+def mx_cast_transposed(x, rms, codes_t, scales_t, eps=0.0, round=ROUND_RCEIL_POW2, layout=SCALES_ROWMAJOR, stream=None):
+    """Column-wise MXCast of x * (1 / (rms + eps)) (rms may be None): codes_t [D, T], scales_t [D, T/32]."""
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mx_cast_transposed(_ptr(x), _ptr(rms), T, D, eps, _ptr(codes_t), _ptr(scales_t), round, layout,
+                                  _stream(stream)), "mx_cast_transposed")

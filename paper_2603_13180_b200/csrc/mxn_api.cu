@@ -167,6 +167,32 @@ mxn_status mxnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block,
                    rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream, mxn::ELEM_E2M1);
 }
 
+mxn_status mx_cast_transposed(const void* x_bf16, const float* rms_or_null, int64_t T, int64_t D, float eps,
+                              void* codes_t_u8, void* scales_t_u8, mxn_round round, mxn_scale_layout layout,
+                              void* cuda_stream)
+{
+    if (T < 0 || D <= 0 || T % 32 != 0 || D % 4 != 0 || D > 0x7FFFFFFF || T / 128 > 65535) return MXN_ERR_SHAPE;
+    if (round < 0 || round > MXN_ROUND_RCEIL_MAX) return MXN_ERR_ENUM;
+    if (layout != MXN_SCALES_ROWMAJOR && layout != MXN_SCALES_SWIZZLE_128x4) return MXN_ERR_ENUM;
+    if (T == 0) return MXN_OK;
+    if (x_bf16 == nullptr || codes_t_u8 == nullptr || scales_t_u8 == nullptr) return MXN_ERR_NULL;
+    if (misaligned(x_bf16, 8) || misaligned(codes_t_u8, 32) || (rms_or_null != nullptr && misaligned(rms_or_null, 4)))
+        return MXN_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (clear_scale_padding(scales_t_u8, D, T / 32, layout, s) != cudaSuccess) return MXN_ERR_CUDA;
+    mxn::TransposedParams P{};
+    P.x = static_cast<const uint16_t*>(x_bf16);
+    P.rms = rms_or_null;
+    P.codes = static_cast<uint8_t*>(codes_t_u8);
+    P.scales = static_cast<uint8_t*>(scales_t_u8);
+    P.T = T;
+    P.D = (int)D;
+    P.eps = eps;
+    P.round = round;
+    P.layout = layout;
+    return mxn::launch_cast_transposed(P, s) == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
+}
+
 mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,
                       const float* rms, int64_t T, int64_t D, void* dx, int dx_is_fp32, float* dgain_f32_or_null,
                       void* workspace, size_t workspace_bytes, void* cuda_stream)

@@ -30,6 +30,19 @@ bool fwd_shape_supported(int64_t D, int B);
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
 cudaError_t read_timeouts(unsigned int* out);
 
+struct TransposedParams {
+    const uint16_t* x;      // bf16 [T, D]
+    const float* rms;       // [T] or nullptr (rho = 1)
+    uint8_t* codes;         // [D, T]
+    uint8_t* scales;        // [D, T/32] row-major or 128x4-tiled (rows = D)
+    int64_t T;
+    int D;
+    float eps;
+    int round, layout;
+    int KT, tiles_per_row;  // filled by the launcher
+};
+cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream);
+
 struct BwdParams {
     const uint16_t* x;      // bf16 [T, D]
     const uint16_t* g;      // bf16 [T, D]

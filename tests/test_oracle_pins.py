@@ -387,6 +387,38 @@ def test_mxfp4_element_format_by_definition(oracle):
     check(codes, scales, bf16_vals(xp), 32)
 
 
+def test_transposed_cast_reduces_to_the_row_cast(oracle):
+    """Blocks along the token axis of X are blocks along the last axis of X^T: without a normaliser the
+    transposed cast equals mx_cast of the transposed matrix; with power-of-two row factors the scaled values
+    stay exact bf16, so the same reduction pins the rho path; general rho is pinned by definition."""
+    x = wl.bits(wl.make_inputs(wl.Workload("t", 96, 160, seed=14, outlier_frac=0.01))["x"])
+    xv = bf16_vals(x)
+    for B in (16, 32):
+        ct, st = oracle.mx_cast_transposed_ref(x, block=B)
+        c, s = oracle.mx_cast_ref(np.ascontiguousarray(x.T), block=B)
+        assert np.array_equal(ct, c) and np.array_equal(st, s)
+    # rho_t = 2^-k_t exactly (r = 2^k, eps = 0): scaled values are exact bf16
+    k = np.random.default_rng(0).integers(-6, 7, size=96)
+    r = np.ldexp(1.0, k).astype(np.float32)
+    ys = bf16_bits(xv * np.ldexp(1.0, -k).astype(np.float32)[:, None])
+    ct, st = oracle.mx_cast_transposed_ref(x, rms=r)
+    c, s = oracle.mx_cast_ref(np.ascontiguousarray(ys.T))
+    assert np.array_equal(ct, c) and np.array_equal(st, s)
+    # general r (the MXNorm estimate) and eps: definitional check
+    _, _, r_est = oracle.mxnorm_ref(x, eps=1e-5)
+    ct, st = oracle.mx_cast_transposed_ref(x, rms=r_est, eps=1e-5)
+    rho = (np.float32(1.0) / (r_est + np.float32(1e-5))).astype(np.float32)
+    y = (xv * rho[:, None]).astype(np.float32).T                      # [D, T]
+    m = np.abs(y).reshape(160, -1, 32).max(-1)
+    sb = smallest_pow2_scale(m)
+    assert np.array_equal(st, sb)
+    code, neg = nearest_code(y.astype(np.float64) / np.repeat(np.ldexp(1.0, sb.astype(int) - 127), 32, axis=1), E4M3_POS)
+    assert np.array_equal(ct, code | (neg.astype(np.uint8) << 7))
+    # zero rms -> rho = 0 -> zero codes, zero scales
+    ct, st = oracle.mx_cast_transposed_ref(x, rms=np.zeros(96, np.float32))
+    assert np.all(st == 0) and np.all((ct & 0x7F) == 0)
+
+
 # ------------------------------------------------------------------ library restatements
 def test_rms_estimate_against_numpy_restatement(oracle):
     x = _rand_rows(7, T=64, D=1024)
