@@ -365,6 +365,31 @@ def main():
         ms4 = time_launches(nvfp4, SETS, args.steps, args.warmup, stream)
         others["mxnorm_nvfp4_fwd"] = {"ms": ms4, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4 / 1e6}
         del o4
+        # MXFP4 (E2M1 codes, E8M0 scales) and the column-wise cast of rho~*X for the weight-gradient GEMM
+        m4 = [mx.alloc_outputs(T, D, 32, layout, nvfp4=True) for _ in range(SETS)]
+
+        def mxfp4(i):
+            c, s, r = m4[i]
+            st = L.mxnorm_mxfp4_fwd(xs[i].data_ptr(), T, D, 32, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(), layout, sh)
+            if st != 0:
+                raise RuntimeError(mx.status_string(st))
+
+        msm4 = time_launches(mxfp4, SETS, args.steps, args.warmup, stream)
+        others["mxnorm_mxfp4_fwd"] = {"ms": msm4, "gbs": (T * D * 2 + T * D // 2 + T * (D // 32) + 4 * T) / msm4 / 1e6}
+        del m4
+        if T % 32 == 0:
+            ct = [torch.empty((D, T), dtype=torch.uint8, device="cuda") for _ in range(SETS)]
+            stt = [torch.empty(mx.scale_bytes(D, T // 32, layout), dtype=torch.uint8, device="cuda") for _ in range(SETS)]
+            r0 = outs[0][2]
+
+            def transposed(i):
+                st = L.mx_cast_transposed(xs[i].data_ptr(), r0.data_ptr(), T, D, EPS, ct[i].data_ptr(), stt[i].data_ptr(), 0, layout, sh)
+                if st != 0:
+                    raise RuntimeError(mx.status_string(st))
+
+            mst = time_launches(transposed, SETS, args.steps, args.warmup, stream)
+            others["mx_cast_transposed"] = {"ms": mst, "gbs": (T * D * 3 + T * D // 32 + 4 * T) / mst / 1e6}
+            del ct, stt
         # backward (C5 tensors: seed 1, gradient ~ N(0, 1e-2), gain)
         w5 = wl.CONFIGS["C5"]
         inp5 = wl.make_inputs(w5) if T == w5.T else wl.make_inputs(w5, T=T)
