@@ -143,6 +143,22 @@ def test_constant_row_closed_form(oracle, a):
     assert np.all(r1 == np.float32(np.float64(np.float32(0.4814)) * abs(av)))
 
 
+def test_epsilon_enters_the_denominator(oracle):
+    # rho~ = 1 / (r~ + eps): with a constant row of ones and eps = 0.5, r~ = 0.4185 and x*rho~ = 1/0.9185 = 1.0887,
+    # which lies in (1,2]: S = 2^(1-8) (biased 120), q = 1.0887*128 = 139.4 -> nearest E4M3 value 144 = 0x71;
+    # r~ itself is reported without eps
+    x = np.full((2, 128), ONE, np.uint16)
+    codes, scales, r = oracle.mxnorm_ref(x, eps=0.5)
+    assert np.all(r == np.float32(0.4185)) and np.all(scales == 120) and np.all(codes == 0x71)
+    codes, scales, r = oracle.mxnorm_nvfp4_ref(x, eps=0.5)
+    # B = 16: x*rho~ = 1/0.9688 = 1.0322; scale = E4M3(1.0322/6 = 0.17203) = 0.171875 = 0x23; q = 6.0055 -> 6 -> 0x77
+    assert np.all(r == np.float32(0.4688)) and np.all(scales == 0x23) and np.all(codes == 0x77)
+    # a zero row stays zero whatever eps is
+    z = np.zeros((1, 64), np.uint16)
+    codes, scales, r = oracle.mxnorm_ref(z, eps=0.5)
+    assert np.all(codes == 0) and np.all(scales == 0) and np.all(r == 0)
+
+
 def test_nvfp4_constant_row_closed_form(oracle):
     x = np.full((2, 64), ONE, np.uint16)
     codes, scales, r = oracle.mxnorm_nvfp4_ref(x)
