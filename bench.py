@@ -362,8 +362,17 @@ def main():
             if st != 0:
                 raise RuntimeError(mx.status_string(st))
 
+        def rms_nvfp4(i):
+            c, s, r = o4[i]
+            st = L.rmsnorm_nvfp4_fwd(xs[i].data_ptr(), T, D, EPS, 1.0, c.data_ptr(), s.data_ptr(), r.data_ptr(), 0, sh)
+            if st != 0:
+                raise RuntimeError(mx.status_string(st))
+
         ms4 = time_launches(nvfp4, SETS, args.steps, args.warmup, stream)
+        ms4r = time_launches(rms_nvfp4, SETS, args.steps, args.warmup, stream)
         others["mxnorm_nvfp4_fwd"] = {"ms": ms4, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4 / 1e6}
+        others["rmsnorm_nvfp4_fwd"] = {"ms": ms4r, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4r / 1e6}
+        result["nvfp4_speedup_vs_rmsnorm_nvfp4_fwd"] = ms4r / ms4
         del o4
         # MXFP4 (E2M1 codes, E8M0 scales) and the column-wise cast of rho~*X for the weight-gradient GEMM
         m4 = [mx.alloc_outputs(T, D, 32, layout, nvfp4=True) for _ in range(SETS)]

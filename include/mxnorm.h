@@ -89,6 +89,13 @@ const char* mxn_status_string(mxn_status s);
  * MXN_ERR_TIMEOUT when it is non-zero (outputs of the affected launch are incomplete), else MXN_OK. */
 mxn_status mxn_device_timeouts(unsigned int* count_out);
 
+/* Diagnostics: the NVFP4 kernels replace the IEEE divisions by 6 and by an E4M3 scale with a multiply and two
+ * fused multiply-adds that give the same correctly rounded quotient.  This call re-checks that claim on the
+ * current device for every binary32 numerator between 2^-100 and 2^100 and every divisor the kernels use
+ * (about a second; it allocates and frees 8 bytes of device memory and synchronises the device - a test
+ * utility, not part of the hot path).  *mismatches_out receives the number of differing quotients (0). */
+mxn_status mxn_selftest_division(unsigned long long* mismatches_out);
+
 /* MXCast - Section 3.2 "Conversion to MXFP8", Eqs. S_tk = cast(m_tk / 256; E8M0),
  * V_tkb = cast(X_tkb / S_tk; E4M3).
  *   x_bf16 [T,D] in; codes_u8 [T,D] out; scales_u8 out (biased E8M0 exponents;
@@ -134,6 +141,13 @@ mxn_status mxnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D,
                             int p, float coef_or_0, float eps, float global_scale,
                             void* codes_u8_packed, void* scales_e4m3, float* rms_est_out_or_null,
                             mxn_scale_layout layout, void* cuda_stream);
+
+/* The conventional path in the NVFP4 format (Algorithm 1's rho from the true RMS, then the same NVFP4 cast as
+ * mxnorm_nvfp4_fwd) - the baseline mxnorm_nvfp4_fwd is compared with, as rmsnorm_mxfp8_fwd is for mxnorm_fwd.
+ * Same buffers and conventions as mxnorm_nvfp4_fwd; rms_out_or_null receives sqrt(mean x^2 + eps). */
+mxn_status rmsnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, float eps, float global_scale,
+                             void* codes_u8_packed, void* scales_e4m3, float* rms_out_or_null,
+                             mxn_scale_layout layout, void* cuda_stream);
 
 /* MXFP4 counterparts of the three forward entry points: E2M1 element values (two per byte, element 2i in
  * the low nibble: codes_u8_packed [T, D/2], 32-byte aligned) with E8M0 block scales, B in {16, 32, 64} -

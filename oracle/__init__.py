@@ -50,6 +50,8 @@ def _load():
         lib.mxnorm_ref.argtypes = [vp, vp, i64, i64, i32, i32, f32, f32, i32, i32, vp, vp, vp]
         lib.mxnorm_nvfp4_ref.argtypes = [vp, i64, i64, i32, f32, f32, f32, vp, vp, vp]
         lib.mxnorm_bwd_ref.argtypes = [vp, vp, vp, vp, i64, i64, vp, vp]
+        lib.rmsnorm_nvfp4_ref.argtypes = [vp, i64, i64, f32, f32, vp, vp, vp]
+        lib.rmsnorm_nvfp4_ref.restype = i32
         lib.mx_cast_transposed_ref.argtypes = [vp, vp, i64, i64, i32, f32, i32, vp, vp]
         lib.mx_cast_transposed_ref.restype = i32
         for f in (lib.mx_cast_ref, lib.rmsnorm_mxfp8_ref, lib.mxnorm_ref, lib.mxnorm_nvfp4_ref,
@@ -150,6 +152,18 @@ def mxnorm_nvfp4_ref(x, p=2, coef=0.0, eps=0.0, global_scale=1.0):
     rms = np.zeros((T,), np.float32)
     _check(_load().mxnorm_nvfp4_ref(_p(x), T, D, p, coef, eps, global_scale,
                                     _p(codes), _p(scales), _p(rms)), "mxnorm_nvfp4_ref")
+    return codes, scales, rms
+
+
+def rmsnorm_nvfp4_ref(x, eps=0.0, global_scale=1.0):
+    """RMSNorm followed by the NVFP4 cast: returns (packed codes [T, D/2] u8, E4M3 scales [T, D/16] u8, rms)."""
+    x = _bf16(x, 2)
+    T, D = x.shape
+    codes = np.zeros((T, D // 2), np.uint8)
+    scales = np.zeros((T, D // 16 if D % 16 == 0 else 0), np.uint8)
+    rms = np.zeros((T,), np.float32)
+    _check(_load().rmsnorm_nvfp4_ref(_p(x), T, D, eps, global_scale, _p(codes), _p(scales), _p(rms)),
+           "rmsnorm_nvfp4_ref")
     return codes, scales, rms
 
 

@@ -364,6 +364,27 @@ int mxnorm_ref(const uint16_t *x_bf16, const uint16_t *gain_bf16, int64_t T, int
 /*     inv_k = fl32(fl32(rho~ * global_scale) / d_k) (0 when d_k = 0);         */
 /*     V_kb = cast(fl32(x_kb * inv_k); E2M1), two codes per byte.              */
 /* ------------------------------------------------------------------------- */
+/* shared NVFP4 tail: given the row's block absmaxes m_k of |x| and rho, emit E4M3 block scales and E2M1 codes */
+static void nvfp4_quantise_row(const uint16_t *xr, const float *m, int64_t D, float rho, float global_scale,
+                               uint8_t *row_codes, uint8_t *row_scales)
+{
+    const int B = 16;
+    int64_t K = D / B;
+    float rho_g = rho * global_scale;
+    for (int64_t k = 0; k < K; ++k) {
+        float a = m[k] * rho;
+        float tk = (a / 6.0f) * global_scale;
+        uint8_t sc = e4m3_encode(tk);
+        row_scales[k] = sc;
+        float dk = e4m3_decode(sc);
+        float inv = dk == 0.0f ? 0.0f : rho_g / dk;
+        for (int b = 0; b < B; ++b) {
+            float q = bf16_to_f32(xr[k * B + b]) * inv;
+            put_code(row_codes, k * B + b, e2m1_encode(q), REF_ELEM_E2M1);
+        }
+    }
+}
+
 int mxnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, int p, float coef, float eps,
                      float global_scale, uint8_t *codes_packed, uint8_t *scales_e4m3,
                      float *rms_est_out)
@@ -378,20 +399,38 @@ int mxnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, int p, float 
         float m[K];
         float r_est, rho;
         mxnorm_row_stat(xr, D, B, p, coef, eps, m, &r_est, &rho);
-        float rho_g = rho * global_scale;
-        for (int64_t k = 0; k < K; ++k) {
-            float a = m[k] * rho;
-            float tk = (a / 6.0f) * global_scale;
-            uint8_t sc = e4m3_encode(tk);
-            scales_e4m3[t * K + k] = sc;
-            float dk = e4m3_decode(sc);
-            float inv = dk == 0.0f ? 0.0f : rho_g / dk;
-            for (int b = 0; b < B; ++b) {
-                float q = bf16_to_f32(xr[k * B + b]) * inv;
-                put_code(codes_packed + t * (D / 2), k * B + b, e2m1_encode(q), REF_ELEM_E2M1);
-            }
-        }
+        nvfp4_quantise_row(xr, m, D, rho, global_scale, codes_packed + t * (D / 2), scales_e4m3 + t * K);
         if (rms_est_out) rms_est_out[t] = r_est;
+    }
+    return 0;
+}
+
+/* The conventional counterpart in the same format: Algorithm 1's rho (true RMS) followed by the NVFP4 cast of
+ * x * rho [reading, as above].  Block absmaxes of fl32(x*rho) equal fl32(m_k * rho) because rounding is monotone. */
+int rmsnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, float eps, float global_scale,
+                      uint8_t *codes_packed, uint8_t *scales_e4m3, float *rms_out)
+{
+    const int B = 16;
+    if (!shape_ok(T, D, B)) return 1;
+    int64_t K = D / B;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *xr = x_bf16 + t * D;
+        float m[K];
+        double ss = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            float mk = 0.0f;
+            for (int b = 0; b < B; ++b) {
+                float v = bf16_to_f32(xr[k * B + b]);
+                ss += (double)v * (double)v;
+                if (fabsf(v) > mk) mk = fabsf(v);
+            }
+            m[k] = mk;
+        }
+        float r = (float)sqrt(ss / (double)D + (double)eps);
+        float rho = r == 0.0f ? 0.0f : 1.0f / r;
+        nvfp4_quantise_row(xr, m, D, rho, global_scale, codes_packed + t * (D / 2), scales_e4m3 + t * K);
+        if (rms_out) rms_out[t] = r;
     }
     return 0;
 }

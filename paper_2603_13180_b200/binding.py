@@ -22,7 +22,7 @@ EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
            "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
-           "mx_cast_transposed")
+           "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -38,6 +38,8 @@ lib.mxn_status_string.argtypes = [_i32]
 lib.mxn_status_string.restype = ctypes.c_char_p
 lib.mxn_device_timeouts.argtypes = [ctypes.POINTER(ctypes.c_uint)]
 lib.mxn_device_timeouts.restype = _i32
+lib.mxn_selftest_division.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
+lib.mxn_selftest_division.restype = _i32
 lib.mx_cast.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _i32, _vp]
 lib.rmsnorm_mxfp8_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
 lib.mxnorm_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
@@ -51,13 +53,14 @@ lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
 lib.mx_cast_fp4.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.rmsnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mxnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.rmsnorm_nvfp4_fwd.argtypes = [_vp, _i64, _i64, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mx_cast_transposed.argtypes = [_vp, _vp, _i64, _i64, _f32, _vp, _vp, _i32, _i32, _vp]
 lib.mxnorm_bwd_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp]
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.argtypes = []
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
 for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
               "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
-           "mx_cast_transposed"):
+           "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division"):
     getattr(lib, _name).restype = _i32
 
 
@@ -97,6 +100,14 @@ def device_timeouts() -> int:
     st = lib.mxn_device_timeouts(ctypes.byref(n))
     if st not in (OK, 7):
         raise MXNormError(st, "mxn_device_timeouts")
+    return int(n.value)
+
+
+def selftest_division() -> int:
+    """Re-checks on the current device that the division shortcuts of the NVFP4 kernels equal IEEE division;
+    returns the number of mismatching quotients (0)."""
+    n = ctypes.c_ulonglong(0)
+    _check(lib.mxn_selftest_division(ctypes.byref(n)), "mxn_selftest_division")
     return int(n.value)
 
 
@@ -215,3 +226,11 @@ def mx_cast_transposed(x, rms, codes_t, scales_t, eps=0.0, round=ROUND_RCEIL_POW
     T, D = x.shape
     _check(lib.mx_cast_transposed(_ptr(x), _ptr(rms), T, D, eps, _ptr(codes_t), _ptr(scales_t), round, layout,
                                   _stream(stream)), "mx_cast_transposed")
+
+
+def rmsnorm_nvfp4_fwd(x, codes_packed, scales_e4m3, rms_out=None, eps=0.0, global_scale=1.0, layout=SCALES_ROWMAJOR,
+                      stream=None):
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.rmsnorm_nvfp4_fwd(_ptr(x), T, D, eps, global_scale, _ptr(codes_packed), _ptr(scales_e4m3), _ptr(rms_out),
+                                 layout, _stream(stream)), "rmsnorm_nvfp4_fwd")

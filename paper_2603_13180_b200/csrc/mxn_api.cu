@@ -114,6 +114,14 @@ mxn_status mxn_device_timeouts(unsigned int* count_out)
     return n == 0 ? MXN_OK : MXN_ERR_TIMEOUT;
 }
 
+mxn_status mxn_selftest_division(unsigned long long* mismatches_out)
+{
+    unsigned long long n = 0;
+    if (mxn::selftest_division(&n) != cudaSuccess) return MXN_ERR_CUDA;
+    if (mismatches_out != nullptr) *mismatches_out = n;
+    return MXN_OK;
+}
+
 mxn_status mx_cast(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8, void* scales_u8,
                    mxn_round round, mxn_scale_layout layout, void* cuda_stream)
 {
@@ -143,6 +151,14 @@ mxn_status mxnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int p, flo
 {
     return run_fwd(mxn::STAT_MX, true, x_bf16, nullptr, T, D, 16, p, coef_or_0, eps, global_scale, codes_u8_packed,
                    scales_e4m3, rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
+}
+
+mxn_status rmsnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, float eps, float global_scale,
+                             void* codes_u8_packed, void* scales_e4m3, float* rms_out_or_null,
+                             mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_fwd(mxn::STAT_RMS, true, x_bf16, nullptr, T, D, 16, 2, 1.0f, eps, global_scale, codes_u8_packed,
+                   scales_e4m3, rms_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
 }
 
 mxn_status mx_cast_fp4(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8_packed, void* scales_u8,

@@ -98,6 +98,38 @@ __device__ __forceinline__ float e4m3_to_f32(uint32_t c)
     return ef ? __uint_as_float(((ef + 120u) << 23) | (mf << 20)) : (float)mf * 0.001953125f;
 }
 
+// ---- correctly rounded division by a known divisor without the division sequence ---------------------
+// q = RN(a*c), r = a - q*d (exact in an FMA), q' = RN(q + r*c) with c = RN(1/d) equals RN(a/d) whenever no
+// intermediate leaves the normal range.  Checked exhaustively on the device (every binary32 numerator with
+// exponent in [2^-100, 2^100)) for d = 6, d = 448 and the eight E4M3 significands 1 + m/8; mxn_selftest_division
+// repeats that check.  Outside the exponent window the IEEE division is used.
+__device__ __forceinline__ bool in_division_window(float a)
+{
+    const uint32_t E = (__float_as_uint(a) >> 23) & 0xFFu;
+    return E - 27u < 200u;   // 2^-100 <= |a| < 2^100
+}
+__device__ __forceinline__ float div_by_known(float a, float d, float c)
+{
+    const float q = __fmul_rn(a, c);
+    const float r = __fmaf_rn(-d, q, a);
+    return __fmaf_rn(r, c, q);
+}
+__device__ __forceinline__ float div_by_6(float a)
+{
+    return in_division_window(a) ? div_by_known(a, 6.0f, 0x1.555556p-3f) : __fdiv_rn(a, 6.0f);
+}
+// RN(1 / (1 + m/8)) for m = 0..7
+__device__ __constant__ float kRcpE4M3Significand[8] = {0x1p+0f, 0x1.c71c72p-1f, 0x1.99999ap-1f, 0x1.745d18p-1f,
+                                                        0x1.555556p-1f, 0x1.3b13b2p-1f, 0x1.24924ap-1f, 0x1.111112p-1f};
+// a / d for d the value of the normal, non-negative E4M3 byte c (exponent field ef >= 1)
+__device__ __forceinline__ float div_by_e4m3_normal(float a, uint32_t code, float d)
+{
+    const uint32_t ef = (code >> 3) & 0xFu, mf = code & 7u;
+    // 1/d = RN(1/(1+mf/8)) * 2^-(ef-7): the power of two is exact
+    const float c = __fmul_rn(kRcpE4M3Significand[mf], __uint_as_float((134u - ef) << 23));
+    return div_by_known(a, d, c);
+}
+
 // ---- E8M0 block scale -----------------------------------------------------------------------
 // biased exponent sb of the power-of-two scale S = 2^(sb-127) for a block whose (normalised)
 // absmax is a >= 0; element format E4M3 (largest power of two 2^8, largest value 448).

@@ -288,6 +288,7 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
                                                      const FwdParams& P, int64_t row, int w, int lane)
 {
     const float rho_g = __fmul_rn(rho, P.global_scale);
+    const bool rho_g_in_window = in_division_window(rho_g);
     uint8_t* cp0 = P.codes + row * (P.D / 2) + (int64_t)(w * kWarp + lane) * 8;
     int64_t soff, sstep;
     scale_addressing<WPR>(P, row, w, lane, soff, sstep);
@@ -297,10 +298,12 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
         const int k = (i * WPR + w) * kWarp + lane;
         // block scale = E4M3(fl32(fl32(a/6) * global_scale)), a = fl32(m * rho~)
         const float a = __fmul_rn(m[i], rho);
-        const float t = __fmul_rn(__fdiv_rn(a, 6.0f), P.global_scale);
+        const float t = __fmul_rn(div_by_6(a), P.global_scale);
         const uint32_t sc = cvt_e4m3x2(t, 0.0f) & 0xFFu;
         const float d = e4m3_to_f32(sc);
-        const float inv = d == 0.0f ? 0.0f : __fdiv_rn(rho_g, d);
+        float inv;
+        if (sc >= 8u && rho_g_in_window) inv = div_by_e4m3_normal(rho_g, sc, d);   // normal scale: no division sequence
+        else inv = d == 0.0f ? 0.0f : __fdiv_rn(rho_g, d);
         uint32_t out[2];
         const float2 ii = make_float2(inv, inv);
 #pragma unroll
@@ -386,7 +389,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxf
     quantise_store_mxfp4<B, NPASS, WPR>(xr, m, rho, P, row, w, lane);
 }
 
-template <int NPASS, int WPR>
+template <int NPASS, int WPR, int STAT>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvfp4_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
@@ -399,10 +402,11 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
     uint32_t xr[NPASS][8];
     float m[NPASS];
     load_row_direct<16, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
-    double stat = block_stats<16, NPASS, STAT_MX>(xr, m, P.p);
+    double stat = block_stats<16, NPASS, STAT>(xr, m, P.p);
+    if (STAT == STAT_RMS) forget_unpacked<NPASS, 8>(xr);
     stat = group_sum<WPR>(stat, group, w, red);
     float r, rho;
-    finish_stat<STAT_MX>(stat, P, r, rho);
+    finish_stat<STAT>(stat, P, r, rho);
     if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     quantise_store_nvfp4<NPASS, WPR>(xr, m, rho, P, row, w, lane);
 }
@@ -497,28 +501,29 @@ static fwd_fn pick_mxfp4_stat(int stat, int wpr, int npass)
     return pick_mxfp4<B, STAT_NONE>(wpr, npass);
 }
 
-template <int NPASS>
+template <int NPASS, int STAT>
 static fwd_fn nvfp4_by_wpr(int wpr)
 {
     switch (wpr) {
-        case 1: return fwd_nvfp4_kernel<NPASS, 1>;
-        case 2: return fwd_nvfp4_kernel<NPASS, 2>;
-        case 3: return fwd_nvfp4_kernel<NPASS, 3>;
-        case 4: return fwd_nvfp4_kernel<NPASS, 4>;
-        case 5: return fwd_nvfp4_kernel<NPASS, 5>;
-        case 6: return fwd_nvfp4_kernel<NPASS, 6>;
-        case 7: return fwd_nvfp4_kernel<NPASS, 7>;
-        case 8: return fwd_nvfp4_kernel<NPASS, 8>;
-        case 16: return fwd_nvfp4_kernel<NPASS, 16>;
+        case 1: return fwd_nvfp4_kernel<NPASS, 1, STAT>;
+        case 2: return fwd_nvfp4_kernel<NPASS, 2, STAT>;
+        case 3: return fwd_nvfp4_kernel<NPASS, 3, STAT>;
+        case 4: return fwd_nvfp4_kernel<NPASS, 4, STAT>;
+        case 5: return fwd_nvfp4_kernel<NPASS, 5, STAT>;
+        case 6: return fwd_nvfp4_kernel<NPASS, 6, STAT>;
+        case 7: return fwd_nvfp4_kernel<NPASS, 7, STAT>;
+        case 8: return fwd_nvfp4_kernel<NPASS, 8, STAT>;
+        case 16: return fwd_nvfp4_kernel<NPASS, 16, STAT>;
         default: return nullptr;
     }
 }
+template <int STAT>
 static fwd_fn pick_nvfp4(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / 16;
-    if (npass == MAXP) return nvfp4_by_wpr<MAXP>(wpr);
-    if (npass == MAXP / 2) return nvfp4_by_wpr<(MAXP >= 2 ? MAXP / 2 : 1)>(wpr);
-    if (npass == 1) return nvfp4_by_wpr<1>(wpr);
+    if (npass == MAXP) return nvfp4_by_wpr<MAXP, STAT>(wpr);
+    if (npass == MAXP / 2) return nvfp4_by_wpr<(MAXP >= 2 ? MAXP / 2 : 1), STAT>(wpr);
+    if (npass == 1) return nvfp4_by_wpr<1, STAT>(wpr);
     return nullptr;
 }
 
@@ -574,7 +579,7 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     const int warps = cta_warps(P.wpr);
     P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
-    if (nvfp4) fn = pick_nvfp4(P.wpr, P.npass);
+    if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
     else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16>(stat, P.wpr, P.npass)
                        : B == 32 ? pick_mxfp4_stat<32>(stat, P.wpr, P.npass) : pick_mxfp4_stat<64>(stat, P.wpr, P.npass);
     else if (B == 16) fn = pick_round<16>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
@@ -595,6 +600,47 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fn, P);
+}
+
+// ---- self test of the division shortcuts ------------------------------------------------------------
+__global__ void selftest_division_kernel(unsigned long long* mismatches)
+{
+    const float divisors[10] = {6.0f, 448.0f, 1.0f, 1.125f, 1.25f, 1.375f, 1.5f, 1.625f, 1.75f, 1.875f};
+    const uint64_t n = (uint64_t)200 << 23;   // exponent fields 27..226, every significand
+    unsigned long long bad = 0;
+    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+        const float a = __uint_as_float((27u << 23) + (uint32_t)i);
+        if (__float_as_uint(div_by_6(a)) != __float_as_uint(__fdiv_rn(a, 6.0f))) ++bad;
+        const float c448 = 0x1.24924ap-9f;
+        if (__float_as_uint(div_by_known(a, 448.0f, c448)) != __float_as_uint(__fdiv_rn(a, 448.0f))) ++bad;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+            // E4M3 codes with exponent fields 1, 7 and 15 and significand m
+            const uint32_t codes[3] = {(1u << 3) | m, (7u << 3) | m, (15u << 3) | (m == 7 ? 6u : m)};
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+                const float d = e4m3_to_f32(codes[j]);
+                if (__float_as_uint(div_by_e4m3_normal(a, codes[j], d)) != __float_as_uint(__fdiv_rn(a, d))) ++bad;
+            }
+        }
+        (void)divisors;
+    }
+    if (bad) atomicAdd(mismatches, bad);
+}
+
+cudaError_t selftest_division(unsigned long long* mismatches_host)
+{
+    unsigned long long* dev = nullptr;
+    cudaError_t e = cudaMalloc(&dev, sizeof(unsigned long long));
+    if (e != cudaSuccess) return e;
+    e = cudaMemset(dev, 0, sizeof(unsigned long long));
+    if (e == cudaSuccess) {
+        selftest_division_kernel<<<148 * 8, 256>>>(dev);
+        e = cudaDeviceSynchronize();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(mismatches_host, dev, sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+    cudaFree(dev);
+    return e;
 }
 
 // number of bounded device-side waits that ran out since the library was loaded (synchronises);

@@ -29,6 +29,7 @@ struct FwdParams {
 bool fwd_shape_supported(int64_t D, int B);
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
 cudaError_t read_timeouts(unsigned int* out);
+cudaError_t selftest_division(unsigned long long* mismatches_host);
 
 struct TransposedParams {
     const uint16_t* x;      // bf16 [T, D]

@@ -4,7 +4,7 @@ folded away; speed-up of `mxnorm_fwd` over the fused conventional path `rmsnorm_
 over the grid.  Both sides are this library's hand-written kernels on the same GPU (the paper compares two
 torch.compile kernels on a GB200).
 
-    python -m paper_2603_13180_b200.sweep [--blocks 32] [--elem e4m3|e2m1] [--tokens 4096 16384 65536] [--json out.json]
+    python -m paper_2603_13180_b200.sweep [--blocks 32] [--elem e4m3|e2m1|nvfp4] [--tokens 4096 16384 65536] [--json out.json]
 """
 from __future__ import annotations
 
@@ -42,7 +42,10 @@ def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4
     for B in blocks:
         for T in tokens:
             for D in hidden:
-                fp4 = elem == "e2m1"
+                nv4 = elem == "nvfp4"
+                if nv4 and B != 16:
+                    continue
+                fp4 = elem == "e2m1" or nv4
                 per_set = T * D * 2 + (T * D // 2 if fp4 else T * D) + T * (D // B) + 4 * T
                 sets = max(2, min(8, -(-3 * l2_bytes // per_set)))        # working set of at least 3x L2
                 g = torch.Generator(device="cuda").manual_seed(T + D)
@@ -51,6 +54,11 @@ def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4
 
                 def mxn(i):
                     c, s, r = outs[i]
+                    if nv4:
+                        st = L.mxnorm_nvfp4_fwd(xs[i].data_ptr(), T, D, 2, 0.0, EPS, 1.0, c.data_ptr(), s.data_ptr(), r.data_ptr(),
+                                                mx.SCALES_SWIZZLE_128x4, sh)
+                        assert st == 0, mx.status_string(st)
+                        return
                     if fp4:
                         st = L.mxnorm_mxfp4_fwd(xs[i].data_ptr(), T, D, B, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
                                                 mx.SCALES_SWIZZLE_128x4, sh)
@@ -62,6 +70,11 @@ def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4
 
                 def rms(i):
                     c, s, r = outs[i]
+                    if nv4:
+                        st = L.rmsnorm_nvfp4_fwd(xs[i].data_ptr(), T, D, EPS, 1.0, c.data_ptr(), s.data_ptr(), r.data_ptr(),
+                                                 mx.SCALES_SWIZZLE_128x4, sh)
+                        assert st == 0, mx.status_string(st)
+                        return
                     if fp4:
                         st = L.rmsnorm_mxfp4_fwd(xs[i].data_ptr(), T, D, B, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(),
                                                  mx.SCALES_SWIZZLE_128x4, sh)
@@ -100,7 +113,8 @@ def main():
     ap.add_argument("--tokens", type=int, nargs="+", default=TOKENS)
     ap.add_argument("--hidden", type=int, nargs="+", default=HIDDEN)
     ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--elem", default="e4m3", choices=["e4m3", "e2m1"], help="element format (E8M0 scales either way)")
+    ap.add_argument("--elem", default="e4m3", choices=["e4m3", "e2m1", "nvfp4"],
+                    help="element format: e4m3/e2m1 with E8M0 scales, or nvfp4 (E2M1 codes, E4M3 scales, block 16)")
     ap.add_argument("--json", default="")
     args = ap.parse_args()
     rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps, elem=args.elem)

@@ -223,3 +223,22 @@ def test_mxfp4_degenerate_rows_and_patterns(binding, oracle):
     codes, scales, r = gu.run_fwd(binding, oracle, "mx4", z)
     gu.assert_exact((codes, scales, r), gu.run_ref(oracle, "mx4", z), "fp4 degenerate")
     assert np.all(scales[3] == 127) and np.all(codes[3] == 0x44)      # constant row closed form
+
+
+@pytest.mark.parametrize("T,D", [(5, 48), (37, 768), (33, 4096), (6, 5120), (3, 16384), (257, 2048)])
+def test_rmsnorm_nvfp4_matches_oracle(binding, oracle, T, D):
+    """The conventional path in NVFP4: r within 1e-6, E4M3 scale bytes and E2M1 codes within the rounding of rho."""
+    x, _ = rows(T, D, seed=17 * T + D)
+    for eps, gs in ((1e-5, 1.0), (0.0, 4.0)):
+        gc, gs_, gr = gu.run_fwd(binding, oracle, "rms_nvfp4", x, eps=eps, global_scale=gs)
+        wc, ws, wr = gu.run_ref(oracle, "rms_nvfp4", x, eps=eps, global_scale=gs)
+        assert np.all(np.abs(gr.astype(np.float64) - wr) <= 1e-6 * np.abs(wr))
+        sdiff = gs_ != ws                                   # an E4M3 scale can move by one code when rho rounds differently
+        assert sdiff.mean() <= 1e-4 and np.all(np.abs(gs_.astype(int) - ws.astype(int)) <= 1)
+        keep = ~np.repeat(sdiff, 16, axis=1)
+        d = gu.nibble_steps(gc, wc)[keep]
+        assert d.max(initial=0) <= 1 and (d != 0).mean() <= 1e-4
+
+
+def test_division_shortcuts_equal_ieee_division(binding):
+    assert binding.selftest_division() == 0

@@ -435,6 +435,30 @@ def test_transposed_cast_reduces_to_the_row_cast(oracle):
     assert np.all(st == 0) and np.all((ct & 0x7F) == 0)
 
 
+def test_rmsnorm_nvfp4_by_definition(oracle):
+    x = wl.bits(wl.make_inputs(wl.Workload("t", 16, 512, seed=21, outlier_frac=0.004))["x"])
+    xv = bf16_vals(x)
+    for gs, eps in ((1.0, 1e-5), (4.0, 0.0)):
+        codes, scales, r = oracle.rmsnorm_nvfp4_ref(x, eps=eps, global_scale=gs)
+        assert np.array_equal(r, oracle.rmsnorm_mxfp8_ref(x, eps=eps)[2])          # same r as Algorithm 1
+        rho = (np.float32(1.0) / r).astype(np.float32)
+        y = (xv * rho[:, None]).astype(np.float32)
+        a = np.abs(y).reshape(16, -1, 16).max(-1)                                # absmax of the normalised values
+        t = ((a / np.float32(6.0)).astype(np.float32) * np.float32(gs)).astype(np.float32)
+        sc, _ = nearest_code(t.astype(np.float64), E4M3_POS)
+        assert np.array_equal(scales, sc)
+        d = E4M3_POS[sc].astype(np.float32)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            inv = np.where(d == 0, np.float32(0), ((rho * np.float32(gs)).astype(np.float32)[:, None] / d).astype(np.float32))
+        q = (xv * np.repeat(inv, 16, axis=1)).astype(np.float32)
+        code, neg = nearest_code(q.astype(np.float64), E2M1_POS)
+        nib = code | (neg.astype(np.uint8) << 3)
+        assert np.array_equal(codes, nib[:, 0::2] | (nib[:, 1::2] << 4))
+    # constant row: RMS = 1, x*rho = 1 -> scale E4M3(1/6 = 0.16667) = 0.171875 (0x23), q = 5.818 -> 6 -> 0x77
+    codes, scales, r = oracle.rmsnorm_nvfp4_ref(np.full((2, 64), ONE, np.uint16))
+    assert np.all(r == 1.0) and np.all(scales == 0x23) and np.all(codes == 0x77)
+
+
 # ------------------------------------------------------------------ library restatements
 def test_rms_estimate_against_numpy_restatement(oracle):
     x = _rand_rows(7, T=64, D=1024)
