@@ -176,6 +176,15 @@ mxn_status mx_cast_transposed(const void* x_bf16, const float* rms_or_null, int6
                               void* codes_t_u8, void* scales_t_u8,
                               mxn_round round, mxn_scale_layout layout, void* cuda_stream);
 
+/* E5M2 casts for gradient tensors (the paper names E4M3 or E5M2 for gradients in the caption of its
+ * computational-graph figure).  OCP E5M2: bias 15, largest finite 57344, largest power of two 2^15, so
+ * S = 2^(ceil(log2 absmax) - 15); codes round-to-nearest-even, saturating; E8M0 scales.  Same buffers,
+ * alignment and layouts as mx_cast / mx_cast_transposed (no normaliser, the paper's rounding rule only). */
+mxn_status mx_cast_e5m2(const void* x_bf16, int64_t T, int64_t D, int block,
+                        void* codes_u8, void* scales_u8, mxn_scale_layout layout, void* cuda_stream);
+mxn_status mx_cast_transposed_e5m2(const void* x_bf16, int64_t T, int64_t D,
+                                   void* codes_t_u8, void* scales_t_u8, mxn_scale_layout layout, void* cuda_stream);
+
 /* Backward - appendix "RMSNorm gradients", used as a straight-through estimator for MXNorm
  * (Section 3.7): the RMSNorm gradient evaluated with the r the forward saved (r~ from
  * mxnorm_fwd, or the true RMS from rmsnorm_mxfp8_fwd - same formula).

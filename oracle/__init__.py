@@ -22,7 +22,7 @@ _SRC = os.path.join(_HERE, "mxnorm_oracle.c")
 _LIB = os.path.join(_HERE, "libmxnorm_oracle.so")
 
 ROUND_RCEIL_POW2, ROUND_FLOOR_OCP, ROUND_RCEIL_MAX = 0, 1, 2
-ELEM_E4M3, ELEM_E2M1 = 0, 1
+ELEM_E4M3, ELEM_E2M1, ELEM_E5M2 = 0, 1, 2
 
 _lib = None
 
@@ -52,7 +52,7 @@ def _load():
         lib.mxnorm_bwd_ref.argtypes = [vp, vp, vp, vp, i64, i64, vp, vp]
         lib.rmsnorm_nvfp4_ref.argtypes = [vp, i64, i64, f32, f32, vp, vp, vp]
         lib.rmsnorm_nvfp4_ref.restype = i32
-        lib.mx_cast_transposed_ref.argtypes = [vp, vp, i64, i64, i32, f32, i32, vp, vp]
+        lib.mx_cast_transposed_ref.argtypes = [vp, vp, i64, i64, i32, f32, i32, i32, vp, vp]
         lib.mx_cast_transposed_ref.restype = i32
         for f in (lib.mx_cast_ref, lib.rmsnorm_mxfp8_ref, lib.mxnorm_ref, lib.mxnorm_nvfp4_ref,
                   lib.mxnorm_bwd_ref):
@@ -69,6 +69,8 @@ def _load():
         lib.mxn_ref_e4m3_decode.restype = f32
         lib.mxn_ref_e2m1_encode.argtypes = [f32]
         lib.mxn_ref_e2m1_encode.restype = ctypes.c_uint8
+        lib.mxn_ref_e5m2_encode.argtypes = [f32]
+        lib.mxn_ref_e5m2_encode.restype = ctypes.c_uint8
         lib.mxn_ref_e8m0_scale.argtypes = [f32, i32, i32]
         lib.mxn_ref_e8m0_scale.restype = ctypes.c_uint8
         lib.mxn_ref_f64_to_bf16.argtypes = [ctypes.c_double]
@@ -182,14 +184,14 @@ def mxnorm_bwd_ref(x, g, gain, rms, want_dx=True, want_dgain=True):
     return dx, dg
 
 
-def mx_cast_transposed_ref(x, rms=None, eps=0.0, block=32, mode=ROUND_RCEIL_POW2):
+def mx_cast_transposed_ref(x, rms=None, eps=0.0, block=32, mode=ROUND_RCEIL_POW2, elem=ELEM_E4M3):
     """Column-wise MXCast of x * rho (rho = 1/(rms+eps), or 1): returns (codes [D, T] u8, scales [D, T/block] u8)."""
     x = _bf16(x, 2)
     T, D = x.shape
     r = None if rms is None else np.ascontiguousarray(rms, dtype=np.float32)
     codes = np.zeros((D, T), np.uint8)
     scales = np.zeros((D, T // block if T % block == 0 else 0), np.uint8)
-    _check(_load().mx_cast_transposed_ref(_p(x), _p(r), T, D, block, eps, mode, _p(codes), _p(scales)),
+    _check(_load().mx_cast_transposed_ref(_p(x), _p(r), T, D, block, eps, mode, elem, _p(codes), _p(scales)),
            "mx_cast_transposed_ref")
     return codes, scales
 
@@ -222,6 +224,10 @@ def e4m3_decode(c: int) -> float:
 
 def e2m1_encode(q: float) -> int:
     return int(_load().mxn_ref_e2m1_encode(q))
+
+
+def e5m2_encode(q: float) -> int:
+    return int(_load().mxn_ref_e5m2_encode(q))
 
 
 def e8m0_scale(a: float, mode=ROUND_RCEIL_POW2, elem=ELEM_E4M3) -> int:

@@ -37,7 +37,7 @@
 
 /* ---- enums (values mirror the public ABI but are declared independently) -- */
 enum { REF_ROUND_RCEIL_POW2 = 0, REF_ROUND_FLOOR_OCP = 1, REF_ROUND_RCEIL_MAX = 2 };
-enum { REF_ELEM_E4M3 = 0, REF_ELEM_E2M1 = 1 };
+enum { REF_ELEM_E4M3 = 0, REF_ELEM_E2M1 = 1, REF_ELEM_E5M2 = 2 };
 
 /* ------------------------------------------------------------------------- */
 /* number formats (MXFP primer appendix; OCP MX element formats)              */
@@ -109,6 +109,33 @@ static float e4m3_decode(uint8_t c)
     return (float)((c & 0x80) ? -v : v);
 }
 
+/* cast(q; E5M2): OCP E5M2 - bias 15, 2 mantissa bits, subnormals down to 2^-16, largest finite 57344
+ * (0x7B); 0x7C is infinity, 0x7D-0x7F NaN.  Round to nearest, ties to even; magnitudes that would round
+ * above 57344 saturate to 57344 [reading: saturating cast]; the sign of zero is kept.  The paper names E5M2
+ * as an option for gradient tensors (caption of the computational-graph figure). */
+static uint8_t e5m2_encode(float q)
+{
+    uint8_t sign = signbit(q) ? 0x80 : 0x00;
+    if (isnan(q)) return sign | 0x7F;
+    double a = fabs((double)q);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return sign | 0x7B;
+    int ex;
+    (void)frexp(a, &ex);
+    int e = ex - 1;                       /* floor(log2 a) */
+    unsigned code;
+    if (e < -14) {                        /* subnormal range: multiples of 2^-16 */
+        code = (unsigned)rint(ldexp(a, 16));   /* 0..4; 4 lands on the smallest normal */
+    } else {
+        double n = rint(ldexp(a, 2 - e)); /* a / 2^(e-2), in [4,8] */
+        if (n == 8.0) { n = 4.0; e += 1; }
+        if (e > 15) return sign | 0x7B;
+        code = ((unsigned)(e + 15) << 2) | ((unsigned)n - 4u);
+    }
+    if (code > 0x7B) code = 0x7B;
+    return sign | (uint8_t)code;
+}
+
 /* cast(q; E2M1): values {0, .5, 1, 1.5, 2, 3, 4, 6}; nibble code 0..7 plus sign
  * in bit 3; round to nearest, ties to the even code; saturate at 6. */
 static uint8_t e2m1_encode(float q)
@@ -138,8 +165,8 @@ static uint8_t e2m1_encode(float q)
 
 /* largest power of two representable by the element format (Algorithm 1/2
  * caption: 256 for E4M3; 4 for E2M1), as a base-2 exponent */
-static int elem_largest_pow2_exp(int elem) { return elem == REF_ELEM_E2M1 ? 2 : 8; }
-static float elem_max(int elem) { return elem == REF_ELEM_E2M1 ? 6.0f : 448.0f; }
+static int elem_largest_pow2_exp(int elem) { return elem == REF_ELEM_E2M1 ? 2 : elem == REF_ELEM_E5M2 ? 15 : 8; }
+static float elem_max(int elem) { return elem == REF_ELEM_E2M1 ? 6.0f : elem == REF_ELEM_E5M2 ? 57344.0f : 448.0f; }
 
 /* ceil(log2 a) and floor(log2 a) of a positive finite binary32, exactly */
 static int ceil_log2f(float a)
@@ -187,7 +214,7 @@ static float inv_scale_f32(uint8_t sb) { return ldexpf(1.0f, 127 - (int)sb); }
 
 static uint8_t elem_encode(float q, int elem)
 {
-    return elem == REF_ELEM_E2M1 ? e2m1_encode(q) : e4m3_encode(q);
+    return elem == REF_ELEM_E2M1 ? e2m1_encode(q) : elem == REF_ELEM_E5M2 ? e5m2_encode(q) : e4m3_encode(q);
 }
 
 /* store one element code: E4M3 one byte per element; E2M1 two per byte,
@@ -481,8 +508,9 @@ int mxnorm_bwd_ref(const uint16_t *x_bf16, const uint16_t *g_bf16, const uint16_
 /*     transposed: codes [D, T], scales [D, T/B].                              */
 /* ------------------------------------------------------------------------- */
 int mx_cast_transposed_ref(const uint16_t *x_bf16, const float *rms_or_null, int64_t T, int64_t D, int B,
-                           float eps, int mode, uint8_t *codes_t, uint8_t *scales_t)
+                           float eps, int mode, int elem, uint8_t *codes_t, uint8_t *scales_t)
 {
+    if (elem == REF_ELEM_E2M1) return 1;   /* one byte per element only */
     if (T < 0 || D <= 0 || !(B == 16 || B == 32 || B == 64) || T % B != 0) return 1;
     int64_t KT = T / B;
 #pragma omp parallel for schedule(static)
@@ -501,10 +529,10 @@ int mx_cast_transposed_ref(const uint16_t *x_bf16, const float *rms_or_null, int
                 float a = fabsf(y[b]);
                 if (a > m) m = a;
             }
-            uint8_t sb = e8m0_scale(m, mode, REF_ELEM_E4M3);
+            uint8_t sb = e8m0_scale(m, mode, elem);
             scales_t[d * KT + k] = sb;
             float inv = inv_scale_f32(sb);
-            for (int b = 0; b < B; ++b) codes_t[d * T + k * B + b] = e4m3_encode(y[b] * inv);
+            for (int b = 0; b < B; ++b) codes_t[d * T + k * B + b] = elem_encode(y[b] * inv, elem);
         }
     }
     return 0;
@@ -533,6 +561,7 @@ int64_t mxn_ref_swizzle_bytes(int64_t T, int64_t K)
 uint8_t mxn_ref_e4m3_encode(float q) { return e4m3_encode(q); }
 float   mxn_ref_e4m3_decode(uint8_t c) { return e4m3_decode(c); }
 uint8_t mxn_ref_e2m1_encode(float q) { return e2m1_encode(q); }
+uint8_t mxn_ref_e5m2_encode(float q) { return e5m2_encode(q); }
 uint8_t mxn_ref_e8m0_scale(float a, int mode, int elem) { return e8m0_scale(a, mode, elem); }
 uint16_t mxn_ref_f64_to_bf16(double v) { return f64_to_bf16(v); }
 

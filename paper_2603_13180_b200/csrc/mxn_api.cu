@@ -183,9 +183,35 @@ mxn_status mxnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block,
                    rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream, mxn::ELEM_E2M1);
 }
 
+namespace {
+mxn_status run_transposed(const void* x_bf16, const float* rms_or_null, int64_t T, int64_t D, float eps, void* codes_t_u8,
+                          void* scales_t_u8, int round, int layout, int elem, void* cuda_stream);
+}
+
+mxn_status mx_cast_e5m2(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8, void* scales_u8,
+                        mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_fwd(mxn::STAT_NONE, false, x_bf16, nullptr, T, D, block, 2, 1.0f, 0.0f, 1.0f, codes_u8, scales_u8, nullptr,
+                   MXN_ROUND_RCEIL_POW2, layout, cuda_stream, mxn::ELEM_E5M2);
+}
+
+mxn_status mx_cast_transposed_e5m2(const void* x_bf16, int64_t T, int64_t D, void* codes_t_u8, void* scales_t_u8,
+                                   mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_transposed(x_bf16, nullptr, T, D, 0.0f, codes_t_u8, scales_t_u8, MXN_ROUND_RCEIL_POW2, layout, mxn::ELEM_E5M2,
+                          cuda_stream);
+}
+
 mxn_status mx_cast_transposed(const void* x_bf16, const float* rms_or_null, int64_t T, int64_t D, float eps,
                               void* codes_t_u8, void* scales_t_u8, mxn_round round, mxn_scale_layout layout,
                               void* cuda_stream)
+{
+    return run_transposed(x_bf16, rms_or_null, T, D, eps, codes_t_u8, scales_t_u8, round, layout, mxn::ELEM_E4M3, cuda_stream);
+}
+
+namespace {
+mxn_status run_transposed(const void* x_bf16, const float* rms_or_null, int64_t T, int64_t D, float eps, void* codes_t_u8,
+                          void* scales_t_u8, int round, int layout, int elem, void* cuda_stream)
 {
     if (T < 0 || D <= 0 || T % 32 != 0 || D % 4 != 0 || D > 0x7FFFFFFF || T / 128 > 65535) return MXN_ERR_SHAPE;
     if (round < 0 || round > MXN_ROUND_RCEIL_MAX) return MXN_ERR_ENUM;
@@ -206,8 +232,10 @@ mxn_status mx_cast_transposed(const void* x_bf16, const float* rms_or_null, int6
     P.eps = eps;
     P.round = round;
     P.layout = layout;
+    P.elem = elem;
     return mxn::launch_cast_transposed(P, s) == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
 }
+}  // namespace
 
 mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,
                       const float* rms, int64_t T, int64_t D, void* dx, int dx_is_fp32, float* dgain_f32_or_null,

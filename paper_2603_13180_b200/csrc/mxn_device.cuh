@@ -76,6 +76,20 @@ __device__ __forceinline__ uint32_t cvt_e4m3x4(float e0, float e1, float e2, flo
         : "=r"(d) : "f"(e0), "f"(e1), "f"(e2), "f"(e3));
     return d;
 }
+// four binary32 -> four E5M2 bytes in memory order (RN-even, saturating to +-57344)
+__device__ __forceinline__ uint32_t cvt_e5m2x4(float e0, float e1, float e2, float e3)
+{
+    uint32_t d;
+    asm("{ .reg .b16 lo, hi; cvt.rn.satfinite.e5m2x2.f32 lo, %2, %1; cvt.rn.satfinite.e5m2x2.f32 hi, %4, %3; mov.b32 %0, {lo, hi}; }"
+        : "=r"(d) : "f"(e0), "f"(e1), "f"(e2), "f"(e3));
+    return d;
+}
+// one byte per element formats: 0 = E4M3 (largest power of two 2^8), 2 = E5M2 (2^15)
+template <int ELEM>
+__device__ __forceinline__ uint32_t cvt_fp8x4(float e0, float e1, float e2, float e3)
+{
+    return ELEM == 2 ? cvt_e5m2x4(e0, e1, e2, e3) : cvt_e4m3x4(e0, e1, e2, e3);
+}
 // two binary32 -> two E2M1 nibbles (RN-even, saturating to +-6); `lo` lands in the low nibble
 __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
 {
@@ -151,12 +165,13 @@ __device__ __forceinline__ uint32_t e8m0_scale(float a, int round)
     return (uint32_t)max(sb, 0);
 }
 // the paper's rule only (round up a/256 to a power of two): sb = max(ceil(log2 a) - 8 + 127, 0)
+template <int EMAX = 8>
 __device__ __forceinline__ uint32_t e8m0_scale_rceil_pow2(float a)
 {
     const uint32_t u = __float_as_uint(a);
     const uint32_t E = u >> 23;
     if (E >= 255u) return (u & 0x7FFFFFu) ? 0u : 254u;   // not finite (outside the contract)
-    const int sb = (int)E + ((u & 0x7FFFFFu) != 0u) - 8;
+    const int sb = (int)E + ((u & 0x7FFFFFu) != 0u) - EMAX;   // EMAX: log2 of the element format's largest power of two
     return (uint32_t)max(sb, 0);
 }
 // 2^(127-sb) as binary32 (sb = 254 gives the subnormal 2^-127)

@@ -142,7 +142,7 @@ __device__ __forceinline__ void scale_addressing(const FwdParams& P, int64_t row
 
 // phase 2 (E4M3 codes, E8M0 scales): scales, codes and their stores for this lane's blocks.
 // PAPER selects the paper's rounding rule at compile time (the common case); otherwise P.round decides.
-template <int B, int NPASS, int WPR, bool GAIN, bool PAPER>
+template <int B, int NPASS, int WPR, bool GAIN, bool PAPER, int ELEM = 0>
 __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][B / 2], const float (&m)[NPASS], float rho,
                                                     const FwdParams& P, int64_t row, int w, int lane)
 {
@@ -161,7 +161,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
         if (!GAIN) {
             // a = fl32(m * rho) is also the absmax of fl32(x * rho): rounding is monotone
             const float a = __fmul_rn(m[i], rho);
-            sb = PAPER ? e8m0_scale_rceil_pow2(a) : e8m0_scale(a, P.round);
+            sb = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(a) : e8m0_scale(a, P.round);
             const float inv = inv_scale(sb);
             // q = fl32(x*rho) * 2^(127-sb).  When neither factor product leaves the normal range the
             // two roundings collapse into the single product x * (rho * 2^(127-sb)).
@@ -172,7 +172,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
 #pragma unroll
                 for (int j = 0; j < W; j += 2) {
                     const float2 q0 = mul2(bf16x2_to_f32x2(xr[i][j]), ff), q1 = mul2(bf16x2_to_f32x2(xr[i][j + 1]), ff);
-                    out[j / 2] = cvt_e4m3x4(q0.x, q0.y, q1.x, q1.y);
+                    out[j / 2] = cvt_fp8x4<ELEM>(q0.x, q0.y, q1.x, q1.y);
                 }
             } else {
                 const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
@@ -180,7 +180,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
                 for (int j = 0; j < W; j += 2) {
                     const float2 q0 = mul2(mul2(bf16x2_to_f32x2(xr[i][j]), rr), ii);
                     const float2 q1 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 1]), rr), ii);
-                    out[j / 2] = cvt_e4m3x4(q0.x, q0.y, q1.x, q1.y);
+                    out[j / 2] = cvt_fp8x4<ELEM>(q0.x, q0.y, q1.x, q1.y);
                 }
             }
         } else {
@@ -206,7 +206,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
                 const float y1 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), bf16_hi(gr[j]));
                 my = fmaxf(my, fmaxf(fabsf(y0), fabsf(y1)));
             }
-            sb = PAPER ? e8m0_scale_rceil_pow2(my) : e8m0_scale(my, P.round);
+            sb = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(my) : e8m0_scale(my, P.round);
             const float inv = inv_scale(sb);
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
@@ -214,7 +214,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
                 const float y1 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), bf16_hi(gr[j]));
                 const float y2 = __fmul_rn(__fmul_rn(bf16_lo(xr[i][j + 1]), rho), bf16_lo(gr[j + 1]));
                 const float y3 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j + 1]), rho), bf16_hi(gr[j + 1]));
-                out[j / 2] = cvt_e4m3x4(__fmul_rn(y0, inv), __fmul_rn(y1, inv), __fmul_rn(y2, inv), __fmul_rn(y3, inv));
+                out[j / 2] = cvt_fp8x4<ELEM>(__fmul_rn(y0, inv), __fmul_rn(y1, inv), __fmul_rn(y2, inv), __fmul_rn(y3, inv));
             }
         }
         if (active) {
@@ -364,6 +364,22 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m
     quantise_store_e4m3<B, NPASS, WPR, GAIN, PAPER>(xr, m, rho, P, row, w, lane);
 }
 
+// plain MXCast to E5M2 codes (gradient tensors), the paper's rounding rule with 2^15
+template <int B, int NPASS, int WPR>
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) cast_e5m2_kernel(const FwdParams P)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / WPR, w = warp - group * WPR;
+    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    pdl_prologue();
+    if (row >= P.T) return;
+    uint32_t xr[NPASS][B / 2];
+    float m[NPASS];
+    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
+    (void)block_stats<B, NPASS, STAT_NONE>(xr, m, 2);
+    quantise_store_e4m3<B, NPASS, WPR, false, true, 2>(xr, m, 1.0f, P, row, w, lane);
+}
+
 // E2M1 codes with E8M0 scales (MXFP4): no gain, the paper's rounding rule
 template <int B, int NPASS, int WPR, int STAT>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxfp4_kernel(const FwdParams P)
@@ -494,6 +510,23 @@ static fwd_fn pick_mxfp4(int wpr, int npass)
     }
 }
 template <int B>
+static fwd_fn pick_e5m2(int wpr, int npass)
+{
+    constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
+    if (wpr == 2) return cast_e5m2_kernel<B, MAXP, 2>;
+    if (wpr == 4) return cast_e5m2_kernel<B, MAXP, 4>;
+    if (wpr == 8) return cast_e5m2_kernel<B, MAXP, 8>;
+    if (wpr == 16) return cast_e5m2_kernel<B, MAXP, 16>;
+    if (wpr != 1) return nullptr;
+    switch (npass) {
+        case 1: return cast_e5m2_kernel<B, 1, 1>;
+        case 2: return cast_e5m2_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1>;
+        case 3: return cast_e5m2_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1>;
+        default: return cast_e5m2_kernel<B, MAXP, 1>;
+    }
+}
+
+template <int B>
 static fwd_fn pick_mxfp4_stat(int stat, int wpr, int npass)
 {
     if (stat == STAT_MX) return pick_mxfp4<B, STAT_MX>(wpr, npass);
@@ -569,7 +602,8 @@ bool fwd_shape_supported(int64_t D, int B)
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
 {
     const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
-    const bool fine = nvfp4 || (!mxfp4 && B == 32 && P.gain == nullptr && P.round == MXN_ROUND_RCEIL_POW2);
+    const bool e5m2 = P.elem == ELEM_E5M2;
+    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && B == 32 && P.gain == nullptr && P.round == MXN_ROUND_RCEIL_POW2);
     if (!plan_row(P.K, B, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
     {
@@ -580,6 +614,7 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
     if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
+    else if (e5m2) fn = B == 16 ? pick_e5m2<16>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32>(P.wpr, P.npass) : pick_e5m2<64>(P.wpr, P.npass);
     else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16>(stat, P.wpr, P.npass)
                        : B == 32 ? pick_mxfp4_stat<32>(stat, P.wpr, P.npass) : pick_mxfp4_stat<64>(stat, P.wpr, P.npass);
     else if (B == 16) fn = pick_round<16>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);

@@ -7,7 +7,7 @@
 namespace mxn {
 
 enum { STAT_NONE = 0, STAT_RMS = 1, STAT_MX = 2 };
-enum { ELEM_E4M3 = 0, ELEM_E2M1 = 1 };
+enum { ELEM_E4M3 = 0, ELEM_E2M1 = 1, ELEM_E5M2 = 2 };
 
 struct FwdParams {
     const uint16_t* x;      // bf16 [T, D]
@@ -40,6 +40,7 @@ struct TransposedParams {
     int D;
     float eps;
     int round, layout;
+    int elem;               // ELEM_E4M3 or ELEM_E5M2
     int KT, tiles_per_row;  // filled by the launcher
 };
 cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream);

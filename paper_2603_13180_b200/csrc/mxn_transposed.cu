@@ -26,7 +26,7 @@ __device__ __forceinline__ uint2 ld_v2(const void* p)
 constexpr int kTrCpl = MXN_TR_CPL;
 constexpr int kTrTileCols = 32 * kTrCpl;
 
-template <bool PAPER>
+template <bool PAPER, int ELEM>
 __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedParams P)
 {
     constexpr int CPL = kTrCpl, WORDS = CPL / 2;
@@ -78,8 +78,8 @@ __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedPa
     float2 inv[WORDS];
 #pragma unroll
     for (int j = 0; j < WORDS; ++j) {
-        sb[2 * j] = PAPER ? e8m0_scale_rceil_pow2(mm[2 * j]) : e8m0_scale(mm[2 * j], P.round);
-        sb[2 * j + 1] = PAPER ? e8m0_scale_rceil_pow2(mm[2 * j + 1]) : e8m0_scale(mm[2 * j + 1], P.round);
+        sb[2 * j] = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(mm[2 * j]) : e8m0_scale(mm[2 * j], P.round);
+        sb[2 * j + 1] = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(mm[2 * j + 1]) : e8m0_scale(mm[2 * j + 1], P.round);
         inv[j] = make_float2(inv_scale(sb[2 * j]), inv_scale(sb[2 * j + 1]));
     }
 
@@ -97,8 +97,8 @@ __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedPa
         }
 #pragma unroll
         for (int j = 0; j < WORDS; ++j) {
-            out[2 * j][r / 4] = cvt_e4m3x4(q[0][j].x, q[1][j].x, q[2][j].x, q[3][j].x);
-            out[2 * j + 1][r / 4] = cvt_e4m3x4(q[0][j].y, q[1][j].y, q[2][j].y, q[3][j].y);
+            out[2 * j][r / 4] = cvt_fp8x4<ELEM>(q[0][j].x, q[1][j].x, q[2][j].x, q[3][j].x);
+            out[2 * j + 1][r / 4] = cvt_fp8x4<ELEM>(q[0][j].y, q[1][j].y, q[2][j].y, q[3][j].y);
         }
     }
     if (!live) return;
@@ -145,7 +145,7 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-template <bool PAPER>
+template <bool PAPER, int ELEM>
 __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_kernel(const TransposedParams P)
 {
     extern __shared__ __align__(128) uint8_t tile_raw[];
@@ -209,8 +209,8 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
                 m1 = fmaxf(m1, fabsf(y.y));
             }
         }
-        const uint32_t sb0 = PAPER ? e8m0_scale_rceil_pow2(m0) : e8m0_scale(m0, P.round);
-        const uint32_t sb1 = PAPER ? e8m0_scale_rceil_pow2(m1) : e8m0_scale(m1, P.round);
+        const uint32_t sb0 = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(m0) : e8m0_scale(m0, P.round);
+        const uint32_t sb1 = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(m1) : e8m0_scale(m1, P.round);
         const float2 inv = make_float2(inv_scale(sb0), inv_scale(sb1));
         uint32_t out0[8], out1[8];
 #pragma unroll
@@ -220,8 +220,8 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
             const float rv[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) q[i] = mul2(mul2(bf16x2_to_f32x2(xr[r + i]), make_float2(rv[i], rv[i])), inv);
-            out0[r / 4] = cvt_e4m3x4(q[0].x, q[1].x, q[2].x, q[3].x);
-            out1[r / 4] = cvt_e4m3x4(q[0].y, q[1].y, q[2].y, q[3].y);
+            out0[r / 4] = cvt_fp8x4<ELEM>(q[0].x, q[1].x, q[2].x, q[3].x);
+            out1[r / 4] = cvt_fp8x4<ELEM>(q[0].y, q[1].y, q[2].y, q[3].y);
         }
         const int c = ctile + (warp * 32 + lane) * 2;
         if (c < P.D) {
@@ -265,7 +265,8 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
     if (P.D % 8 == 0) {   // 16-byte row chunks: the shared-memory staged kernel
         const int64_t sx = (P.D + kTsCols - 1) / kTsCols, sy = (P.T / 32 + kTsTpc - 1) / kTsTpc;
         if (sy <= 65535) {
-            auto kfn = P.round == MXN_ROUND_RCEIL_POW2 ? cast_transposed_smem_kernel<true> : cast_transposed_smem_kernel<false>;
+            auto kfn = P.elem == ELEM_E5M2 ? cast_transposed_smem_kernel<true, 2>
+                       : P.round == MXN_ROUND_RCEIL_POW2 ? cast_transposed_smem_kernel<true, 0> : cast_transposed_smem_kernel<false, 0>;
             const int smem = kTsStages * kTsStageBytes;
             const cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
             if (e != cudaSuccess) return e;
@@ -276,8 +277,9 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
         }
     }
 #endif
-    if (P.round == MXN_ROUND_RCEIL_POW2) return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<true>, P);
-    return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<false>, P);
+    if (P.elem == ELEM_E5M2) return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<true, 2>, P);
+    if (P.round == MXN_ROUND_RCEIL_POW2) return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<true, 0>, P);
+    return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<false, 0>, P);
 }
 
 }  // namespace mxn

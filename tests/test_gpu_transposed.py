@@ -83,3 +83,48 @@ def test_transposed_cast_argument_errors(binding):
     assert L.mx_cast_transposed(None, None, 128, 128, 0.0, fake, fake, 0, 0, None) == 1
     assert L.mx_cast_transposed(fake + 4, None, 128, 128, 0.0, fake, fake, 0, 0, None) == 3
     assert L.mx_cast_transposed(fake, None, 128, 128, 0.0, fake, fake, 5, 0, None) == 4
+
+
+@pytest.mark.parametrize("T,D", [(64, 128), (96, 160), (256, 4096), (160, 132)])
+def test_e5m2_casts_match_oracle_bit_for_bit(binding, oracle, T, D):
+    """E5M2 codes (gradient tensors): row-wise and column-wise casts."""
+    inp = wl.make_inputs(wl.Workload("t", T, D, seed=3 * T + D, outlier_frac=0.01, has_grad=True))
+    g = wl.bits(inp["grad"])
+    x = wl.from_bits(g).cuda()
+    # column-wise
+    cfull, codes = gu.guarded(D * T)
+    sfull, scales = gu.guarded(binding.scale_bytes(D, T // 32, 0))
+    binding.mx_cast_transposed_e5m2(x, codes, scales)
+    torch.cuda.synchronize()
+    assert gu.guards_intact(cfull, D * T) and gu.guards_intact(sfull, D * (T // 32))
+    wc, ws = oracle.mx_cast_transposed_ref(g, elem=oracle.ELEM_E5M2)
+    assert np.array_equal(scales.cpu().numpy().reshape(D, T // 32), ws)
+    assert np.array_equal(codes.cpu().numpy().reshape(D, T), wc)
+    # row-wise, all block sizes that divide D
+    for B in (16, 32, 64):
+        if D % B:
+            continue
+        cfull, codes = gu.guarded(T * D)
+        sfull, scales = gu.guarded(T * (D // B))
+        binding.mx_cast_e5m2(x, codes, scales, block=B)
+        torch.cuda.synchronize()
+        assert gu.guards_intact(cfull, T * D) and gu.guards_intact(sfull, T * (D // B))
+        wc, ws = oracle.mx_cast_ref(g, block=B, elem=oracle.ELEM_E5M2)
+        assert np.array_equal(scales.cpu().numpy().reshape(T, D // B), ws)
+        assert np.array_equal(codes.cpu().numpy().reshape(T, D), wc)
+
+
+def test_e5m2_all_bf16_patterns(binding, oracle):
+    pats = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    pats = pats[(pats & 0x7F80) != 0x7F80]
+    xb = np.zeros((pats.size, 32), np.uint16)
+    xb[:, 0] = pats
+    xb[:, 9] = (pats >> 1) & 0x7FFF
+    xb[(xb[:, 9] & 0x7F80) == 0x7F80, 9] = 0
+    x = wl.from_bits(xb).cuda()
+    codes = torch.empty((pats.size, 32), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((pats.size,), dtype=torch.uint8, device="cuda")
+    binding.mx_cast_e5m2(x, codes, scales)
+    torch.cuda.synchronize()
+    wc, ws = oracle.mx_cast_ref(xb, elem=oracle.ELEM_E5M2)
+    assert np.array_equal(scales.cpu().numpy().reshape(-1, 1), ws) and np.array_equal(codes.cpu().numpy(), wc)

@@ -459,6 +459,46 @@ def test_rmsnorm_nvfp4_by_definition(oracle):
     assert np.all(r == 1.0) and np.all(scales == 0x23) and np.all(codes == 0x77)
 
 
+E5M2_POS = np.array([(m * 2.0 ** -16) if e == 0 else (4 + m) * 2.0 ** (e - 17)
+                     for e in range(32) for m in range(4)][:0x7C], dtype=np.float64)   # codes 0..0x7B (57344)
+
+
+def test_e5m2_element_format(oracle):
+    """E5M2 (an option the paper names for gradients): encoder against brute force and torch's cast; the cast uses
+    2^15, the largest power of two of the format, so block maxima land in (2^14, 2^15]."""
+    assert E5M2_POS[-1] == 57344.0 and E5M2_POS[4] == 2.0 ** -14
+    g = E5M2_POS
+    mids = (g[:-1] + g[1:]) / 2
+    probes = np.concatenate([g, mids, np.nextafter(mids.astype(np.float32), np.float32(0)),
+                             np.nextafter(mids.astype(np.float32), np.float32(1e9)), [57344.0, 60000.0, 61440.0, 1e6, 2.0 ** -17, 1e-30]])
+    probes = probes.astype(np.float32)
+    want, _ = nearest_code(probes.astype(np.float64), g)
+    got = np.array([oracle.e5m2_encode(float(v)) for v in probes], np.uint8)
+    assert np.array_equal(got, want)
+    assert oracle.e5m2_encode(-3.0) == (0x80 | oracle.e5m2_encode(3.0)) and oracle.e5m2_encode(float("inf")) == 0x7B
+    rng = np.random.default_rng(0)
+    v = np.concatenate([rng.standard_normal(20000) * 1000, rng.standard_normal(20000), rng.standard_normal(5000) * 1e-4]).astype(np.float32)
+    v = v[np.abs(v) <= 57344.0]
+    want = torch.from_numpy(v).to(torch.float8_e5m2).view(torch.uint8).numpy()
+    got = np.array([oracle.e5m2_encode(float(a)) for a in v], np.uint8)
+    assert np.array_equal(got, want)
+    # the cast by definition
+    x = wl.bits(wl.make_inputs(wl.Workload("t", 32, 256, seed=31, outlier_frac=0.01))["x"])
+    xv = bf16_vals(x)
+    codes, scales = oracle.mx_cast_ref(x, elem=oracle.ELEM_E5M2)
+    m = np.abs(xv).reshape(32, -1, 32).max(-1)
+    sb = smallest_pow2_scale(m, emax=15)
+    assert np.array_equal(scales, sb)
+    S = np.repeat(np.ldexp(1.0, sb.astype(int) - 127), 32, axis=1)
+    code, neg = nearest_code(xv.astype(np.float64) / S, g)
+    assert np.array_equal(codes, code | (neg.astype(np.uint8) << 7))
+    top = (codes & 0x7F).reshape(32, -1, 32).max(-1)
+    assert np.all((top >= 0x74) & (top <= 0x78))     # (2^14, 2^15], where values just above 2^14 round down to it
+    ct, st = oracle.mx_cast_transposed_ref(x, elem=oracle.ELEM_E5M2)
+    c2, s2 = oracle.mx_cast_ref(np.ascontiguousarray(x.T), elem=oracle.ELEM_E5M2)
+    assert np.array_equal(ct, c2) and np.array_equal(st, s2)
+
+
 # ------------------------------------------------------------------ library restatements
 def test_rms_estimate_against_numpy_restatement(oracle):
     x = _rand_rows(7, T=64, D=1024)
