@@ -129,6 +129,18 @@ mxn_status mxnorm_fwd(const void* x_bf16, const void* gain_bf16_or_null,
                       void* codes_u8, void* scales_u8, float* rms_est_out_or_null,
                       mxn_round round, mxn_scale_layout layout, void* cuda_stream);
 
+/* Post-round MXNorm - appendix "Post-round MXNorm" (the paper's ablation; it reports this variant unstable at
+ * 8B parameters): the RMS is estimated from the block absmaxes after rounding them to powers of two,
+ *   xbar = (1/K) sum_k 2^floor(log2 m_k),  r~ = f^-1(xbar),  f(sigma) = E[max_i 2^floor(log2 |X_i|)] for a block
+ *   of B i.i.d. N(0, sigma^2) values; f^-1 by linear interpolation in a table of f^-1(2^(i/64)), i = 0..64, on
+ *   [1,2] and f^-1(x) = 2^-k f^-1(2^k x) elsewhere (the table size is this library's choice).
+ * Scales and codes then follow mxnorm_fwd with this r~ (no gain, the paper's rounding rule, B in {16,32,64}).
+ * The first call for a block size on a device computes the table on the host (tens of milliseconds) and copies
+ * it to constant memory - a synchronous copy: make that call outside stream capture. */
+mxn_status mxnorm_postround_fwd(const void* x_bf16, int64_t T, int64_t D, int block, float eps,
+                                void* codes_u8, void* scales_u8, float* rms_est_out_or_null,
+                                mxn_scale_layout layout, void* cuda_stream);
+
 /* NVFP4 variant of MXNorm (the paper benchmarks "B = 16, E2M1" in Section 4.3 but does not
  * define the scale rule; this is the usual NVFP4 convention).
  *   B = 16; r~ and rho~ as in mxnorm_fwd with the (16, p) constant (0.4688 for p = 2);

@@ -52,6 +52,12 @@ def _load():
         lib.mxnorm_bwd_ref.argtypes = [vp, vp, vp, vp, i64, i64, vp, vp]
         lib.rmsnorm_nvfp4_ref.argtypes = [vp, i64, i64, f32, f32, vp, vp, vp]
         lib.rmsnorm_nvfp4_ref.restype = i32
+        lib.mxnorm_postround_ref.argtypes = [vp, i64, i64, i32, f32, i32, vp, vp, vp]
+        lib.mxnorm_postround_ref.restype = i32
+        lib.mxn_ref_postround_f.argtypes = [ctypes.c_double, i32]
+        lib.mxn_ref_postround_f.restype = ctypes.c_double
+        lib.mxn_ref_postround_f_inverse.argtypes = [ctypes.c_double, i32]
+        lib.mxn_ref_postround_f_inverse.restype = ctypes.c_double
         lib.mx_cast_transposed_ref.argtypes = [vp, vp, i64, i64, i32, f32, i32, i32, vp, vp]
         lib.mx_cast_transposed_ref.restype = i32
         for f in (lib.mx_cast_ref, lib.rmsnorm_mxfp8_ref, lib.mxnorm_ref, lib.mxnorm_nvfp4_ref,
@@ -167,6 +173,26 @@ def rmsnorm_nvfp4_ref(x, eps=0.0, global_scale=1.0):
     _check(_load().rmsnorm_nvfp4_ref(_p(x), T, D, eps, global_scale, _p(codes), _p(scales), _p(rms)),
            "rmsnorm_nvfp4_ref")
     return codes, scales, rms
+
+
+def mxnorm_postround_ref(x, eps=0.0, block=32, mode=ROUND_RCEIL_POW2):
+    """Post-round MXNorm (RMS from the power-of-two-rounded block absmaxes): returns (codes, scales, rms_estimate)."""
+    x = _bf16(x, 2)
+    T, D = x.shape
+    codes = np.zeros((T, D), np.uint8)
+    scales = np.zeros((T, D // block if D % block == 0 else 0), np.uint8)
+    rms = np.zeros((T,), np.float32)
+    _check(_load().mxnorm_postround_ref(_p(x), T, D, block, eps, mode, _p(codes), _p(scales), _p(rms)),
+           "mxnorm_postround_ref")
+    return codes, scales, rms
+
+
+def postround_f(sigma: float, block: int) -> float:
+    return float(_load().mxn_ref_postround_f(sigma, block))
+
+
+def postround_f_inverse(x: float, block: int) -> float:
+    return float(_load().mxn_ref_postround_f_inverse(x, block))
 
 
 def mxnorm_bwd_ref(x, g, gain, rms, want_dx=True, want_dgain=True):

@@ -499,6 +499,101 @@ int mxnorm_bwd_ref(const uint16_t *x_bf16, const uint16_t *g_bf16, const uint16_
 }
 
 /* ------------------------------------------------------------------------- */
+/* O7  Post-round MXNorm (appendix "Post-round MXNorm"): the RMS is estimated    */
+/*     from the block absmaxes AFTER rounding them to powers of two,            */
+/*       s_k = r(m_k) = 2^floor(log2 m_k)   (0 for a zero block),                */
+/*       xbar = (1/K) sum_k s_k,   r~ = f^-1(xbar),                              */
+/*     where f(sigma) = E[max_i r(X_i)] for B i.i.d. N(0, sigma^2) values:       */
+/*       f(sigma) = sum_j 2^j [ P(2^(j+1)) - P(2^j) ],  P(t) = erf(t/(sigma sqrt2))^B */
+/*     [reading: the printed series has the two terms in the other order, which  */
+/*     would make the expectation negative].  f^-1 is evaluated as the appendix  */
+/*     describes: a table of f^-1(2^(i/A)), i = 0..A, linear interpolation in x  */
+/*     on [1,2], and f^-1(x) = 2^-k f^-1(2^k x) elsewhere [reading: A = 64; the  */
+/*     paper leaves A open].  Scales and codes then follow Algorithm 2 with this */
+/*     r~.  PARITY UNPINNED by printed values: pinned by f(2s) = 2f(s), a Monte  */
+/*     Carlo estimate of f, f^-1(f(s)) = s and the estimator's mean on Gaussian  */
+/*     rows.                                                                     */
+/* ------------------------------------------------------------------------- */
+#define POSTROUND_A 64
+
+static double postround_f(double sigma, int B)
+{
+    /* terms are negligible below 2^-60 sigma (P ~ 0) and above 2^5 sigma (P(2^j) = 1 to the last bit) */
+    int j0 = (int)floor(log2(sigma));
+    double sum = 0.0;
+    for (int j = j0 - 64; j <= j0 + 6; ++j) {
+        double lo = erf(ldexp(1.0, j) / (sigma * 1.4142135623730951));
+        double hi = erf(ldexp(1.0, j + 1) / (sigma * 1.4142135623730951));
+        sum += ldexp(1.0, j) * (pow(hi, B) - pow(lo, B));
+    }
+    return sum;
+}
+
+static double postround_f_inverse(double x, int B)
+{
+    /* f is increasing and f(sigma) lies between 0.5 sigma and 4 sigma for B in 16..64: bisect */
+    double lo = x / 8.0, hi = x * 4.0;
+    for (int it = 0; it < 200; ++it) {
+        double mid = 0.5 * (lo + hi);
+        if (postround_f(mid, B) < x) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+static void postround_table(int B, double *nodes, double *values)
+{
+    for (int i = 0; i <= POSTROUND_A; ++i) {
+        nodes[i] = exp2((double)i / POSTROUND_A);
+        values[i] = postround_f_inverse(nodes[i], B);
+    }
+    nodes[POSTROUND_A] = 2.0;
+}
+
+static double postround_estimate(double xbar, const double *nodes, const double *values)
+{
+    if (!(xbar > 0.0)) return 0.0;
+    int ex;
+    double z = 2.0 * frexp(xbar, &ex); /* xbar = z * 2^(ex-1), z in [1,2) */
+    int i = 0;
+    while (i + 1 < POSTROUND_A && nodes[i + 1] <= z) ++i; /* nodes[i] <= z < nodes[i+1] */
+    double v = values[i] + (z - nodes[i]) * ((values[i + 1] - values[i]) / (nodes[i + 1] - nodes[i]));
+    return ldexp(v, ex - 1);
+}
+
+double mxn_ref_postround_f(double sigma, int B) { return postround_f(sigma, B); }
+double mxn_ref_postround_f_inverse(double x, int B) { return postround_f_inverse(x, B); }
+
+int mxnorm_postround_ref(const uint16_t *x_bf16, int64_t T, int64_t D, int B, float eps, int mode,
+                         uint8_t *codes, uint8_t *scales, float *rms_est_out)
+{
+    if (!shape_ok(T, D, B)) return 1;
+    int64_t K = D / B;
+    double nodes[POSTROUND_A + 1], values[POSTROUND_A + 1];
+    postround_table(B, nodes, values);
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *xr = x_bf16 + t * D;
+        float y[D];
+        double s = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            float mk = 0.0f;
+            for (int b = 0; b < B; ++b) {
+                float a = fabsf(bf16_to_f32(xr[k * B + b]));
+                if (a > mk) mk = a;
+            }
+            if (mk > 0.0f) s += ldexp(1.0, floor_log2f(mk));
+        }
+        float rt = (float)postround_estimate(s / (double)K, nodes, values);
+        float den = rt + eps;
+        float rho = den == 0.0f ? 0.0f : 1.0f / den;
+        for (int64_t d = 0; d < D; ++d) y[d] = bf16_to_f32(xr[d]) * rho;
+        quantise_row(y, D, B, mode, REF_ELEM_E4M3, codes + t * D, scales + t * K);
+        if (rms_est_out) rms_est_out[t] = rt;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* O6  Column-wise (transposed) MXCast for the weight-gradient GEMM            */
 /*     (Section "MXNormLinear": grad W = MXCast(grad H^T) MXCast(rho~ X) gamma,*/
 /*     where the activation must be block-quantised along the TOKEN axis).     */

@@ -23,7 +23,7 @@ EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
            "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
-           "mx_cast_e5m2", "mx_cast_transposed_e5m2")
+           "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -54,6 +54,7 @@ lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
 lib.mx_cast_fp4.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.rmsnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mxnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.mxnorm_postround_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mx_cast_e5m2.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.mx_cast_transposed_e5m2.argtypes = [_vp, _i64, _i64, _vp, _vp, _i32, _vp]
 lib.rmsnorm_nvfp4_fwd.argtypes = [_vp, _i64, _i64, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
@@ -64,7 +65,7 @@ lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
 for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
               "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
-           "mx_cast_e5m2", "mx_cast_transposed_e5m2"):
+           "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd"):
     getattr(lib, _name).restype = _i32
 
 
@@ -251,3 +252,11 @@ def mx_cast_transposed_e5m2(x, codes_t, scales_t, layout=SCALES_ROWMAJOR, stream
     T, D = x.shape
     _check(lib.mx_cast_transposed_e5m2(_ptr(x), T, D, _ptr(codes_t), _ptr(scales_t), layout, _stream(stream)),
            "mx_cast_transposed_e5m2")
+
+
+def mxnorm_postround_fwd(x, codes, scales, rms_est_out=None, eps=0.0, block=32, layout=SCALES_ROWMAJOR, stream=None):
+    """MXNorm with the RMS estimated from power-of-two-rounded block absmaxes (the paper's ablation)."""
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mxnorm_postround_fwd(_ptr(x), T, D, block, eps, _ptr(codes), _ptr(scales), _ptr(rms_est_out), layout,
+                                    _stream(stream)), "mxnorm_postround_fwd")

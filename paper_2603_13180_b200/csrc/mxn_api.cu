@@ -161,6 +161,16 @@ mxn_status rmsnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, float eps
                    scales_e4m3, rms_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
 }
 
+mxn_status mxnorm_postround_fwd(const void* x_bf16, int64_t T, int64_t D, int block, float eps, void* codes_u8,
+                                void* scales_u8, float* rms_est_out_or_null, mxn_scale_layout layout, void* cuda_stream)
+{
+    mxn_status st = check_common(x_bf16, T, D, block, codes_u8, scales_u8, MXN_ROUND_RCEIL_POW2, layout);
+    if (st != MXN_OK || T == 0) return st;
+    if (mxn::postround_prepare(block) != cudaSuccess) return MXN_ERR_CUDA;
+    return run_fwd(mxn::STAT_POSTROUND, false, x_bf16, nullptr, T, D, block, 2, 1.0f, eps, 1.0f, codes_u8, scales_u8,
+                   rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
+}
+
 mxn_status mx_cast_fp4(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8_packed, void* scales_u8,
                        mxn_scale_layout layout, void* cuda_stream)
 {

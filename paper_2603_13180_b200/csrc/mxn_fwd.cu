@@ -11,6 +11,9 @@
 //   * the only cross-lane step is the row statistic: K = D/B block values (MXNorm) instead of
 //     D squares (RMSNorm), reduced in binary64 by shuffles (and through shared memory when a row
 //     spans several warps).
+#include <cmath>
+#include <mutex>
+
 #include "mxn_device.cuh"
 #include "mxn_internal.h"
 
@@ -30,6 +33,29 @@ namespace mxn {
 __host__ __device__ constexpr int rows_per_cta(int wpr) { return MXN_FWD_WARPS / wpr > 1 ? MXN_FWD_WARPS / wpr : 1; }
 __host__ __device__ constexpr int cta_warps(int wpr) { return wpr * rows_per_cta(wpr); }
 
+// ---- post-round estimator tables (appendix "Post-round MXNorm") ------------------------------------
+// f^-1 sampled at the 65 nodes 2^(i/64) of [1,2] for each block size, with the slope of every interval;
+// filled by postround_prepare() on the host, read by finish_stat<STAT_POSTROUND>.
+constexpr int kPrIntervals = 64;
+__device__ __constant__ double c_pr_nodes[kPrIntervals + 1];
+__device__ __constant__ double c_pr_values[3][kPrIntervals + 1];
+__device__ __constant__ double c_pr_slopes[3][kPrIntervals];
+
+__device__ __forceinline__ double postround_estimate(double xbar, int table)
+{
+    if (!(xbar > 0.0)) return 0.0;
+    const unsigned long long bits = (unsigned long long)__double_as_longlong(xbar);
+    const int e = (int)((bits >> 52) & 0x7FFull) - 1023;
+    const double z = __longlong_as_double((long long)((bits & 0x000FFFFFFFFFFFFFull) | 0x3FF0000000000000ull));   // in [1,2)
+    int i = 0;
+#pragma unroll
+    for (int step = kPrIntervals / 2; step >= 1; step >>= 1)
+        if (c_pr_nodes[i + step] <= z) i += step;        // nodes[i] <= z < nodes[i+1]
+    const double v = __dadd_rn(c_pr_values[table][i], __dmul_rn(__dadd_rn(z, -c_pr_nodes[i]), c_pr_slopes[table][i]));
+    const double pow2 = __longlong_as_double((long long)(unsigned long long)(e + 1023) << 52);
+    return __dmul_rn(v, pow2);
+}
+
 // row statistic -> (r, rho) ; one value per row group ------------------------------------------
 template <int STAT>
 __device__ __forceinline__ void finish_stat(double s, const FwdParams& P, float& r, float& rho)
@@ -40,6 +66,12 @@ __device__ __forceinline__ void finish_stat(double s, const FwdParams& P, float&
         double mean = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.K);
         double G = P.p == 2 ? __dsqrt_rn(mean) : mean;
         r = __double2float_rn(__dmul_rn((double)P.coef, G));
+        float den = __fadd_rn(r, P.eps);
+        rho = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
+    } else if (STAT == STAT_POSTROUND) {
+        // xbar = mean of the power-of-two-rounded block absmaxes; r~ = f^-1(xbar); rho~ = 1 / fl32(r~ + eps)
+        const double xbar = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.K);
+        r = __double2float_rn(postround_estimate(xbar, P.pr_table));
         float den = __fadd_rn(r, P.eps);
         rho = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
     } else if (STAT == STAT_RMS) {
@@ -101,6 +133,8 @@ __device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2]
             double md = (double)m[i];
             stat = p == 2 ? __fma_rn(md, md, stat) : __dadd_rn(stat, md);   // m^2 is exact in binary64
         }
+        if (STAT == STAT_POSTROUND)   // 2^floor(log2 m): the absmax with its significand cleared (0 stays 0)
+            stat = __dadd_rn(stat, (double)__uint_as_float(__float_as_uint(m[i]) & 0x7F800000u));
         if (STAT == STAT_RMS) {
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
@@ -465,7 +499,7 @@ template <int B, int STAT, bool GAIN, bool PAPER>
 static fwd_fn pick_e4m3(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    constexpr bool FINE = B == 32 && !GAIN && PAPER;
+    constexpr bool FINE = B == 32 && !GAIN && PAPER && STAT != STAT_POSTROUND;
     if (FINE || wpr > 1) {
         if (npass == MAXP) return e4m3_by_wpr<B, MAXP, STAT, GAIN, PAPER, FINE>(wpr);
         if (FINE && npass == 1) return e4m3_by_wpr<B, 1, STAT, GAIN, PAPER, FINE>(wpr);
@@ -485,6 +519,7 @@ static fwd_fn pick_stat(int stat, bool gain, int wpr, int npass)
         case STAT_NONE: return pick_e4m3<B, STAT_NONE, false, PAPER>(wpr, npass);
         case STAT_RMS: return gain ? pick_e4m3<B, STAT_RMS, true, PAPER>(wpr, npass) : pick_e4m3<B, STAT_RMS, false, PAPER>(wpr, npass);
         case STAT_MX: return gain ? pick_e4m3<B, STAT_MX, true, PAPER>(wpr, npass) : pick_e4m3<B, STAT_MX, false, PAPER>(wpr, npass);
+        case STAT_POSTROUND: return (gain || !PAPER) ? nullptr : pick_e4m3<B, STAT_POSTROUND, false, true>(wpr, npass);
         default: return nullptr;
     }
 }
@@ -603,7 +638,9 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
 {
     const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
     const bool e5m2 = P.elem == ELEM_E5M2;
-    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && B == 32 && P.gain == nullptr && P.round == MXN_ROUND_RCEIL_POW2);
+    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && stat != STAT_POSTROUND && B == 32 && P.gain == nullptr &&
+                                P.round == MXN_ROUND_RCEIL_POW2);
+    P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
     if (!plan_row(P.K, B, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
     {
@@ -635,6 +672,55 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fn, P);
+}
+
+// ---- host side of the post-round estimator: f, its inverse and the table --------------------------
+// f(sigma) = E[max_i 2^floor(log2 |X_i|)] for B i.i.d. N(0, sigma^2) values
+//          = sum_j 2^j (P(2^(j+1)) - P(2^j)),  P(t) = erf(t / (sigma sqrt 2))^B.
+static double pr_expected_rounded_max(double sigma, int B)
+{
+    const double inv = 1.0 / (sigma * std::sqrt(2.0));
+    const int centre = (int)std::floor(std::log2(sigma));
+    double total = 0.0, below = std::pow(std::erf(std::ldexp(1.0, centre - 64) * inv), B);
+    for (int j = centre - 64; j <= centre + 6; ++j) {
+        const double above = std::pow(std::erf(std::ldexp(1.0, j + 1) * inv), B);
+        total += std::ldexp(1.0, j) * (above - below);
+        below = above;
+    }
+    return total;
+}
+static double pr_invert(double x, int B)
+{
+    double a = x / 8.0, b = x * 4.0;   // f(sigma) lies between sigma/2 and 4 sigma for these block sizes
+    for (int it = 0; it < 200; ++it) {
+        const double mid = 0.5 * (a + b);
+        (pr_expected_rounded_max(mid, B) < x ? a : b) = mid;
+    }
+    return 0.5 * (a + b);
+}
+
+cudaError_t postround_prepare(int B)
+{
+    static std::mutex mtx;
+    static bool done[64][3] = {};
+    const int table = B == 16 ? 0 : B == 32 ? 1 : 2;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mtx);
+    if (done[dev][table]) return cudaSuccess;
+    double nodes[kPrIntervals + 1], values[kPrIntervals + 1], slopes[kPrIntervals];
+    for (int i = 0; i <= kPrIntervals; ++i) {
+        nodes[i] = i == kPrIntervals ? 2.0 : std::exp2((double)i / kPrIntervals);
+        values[i] = pr_invert(nodes[i], B);
+    }
+    for (int i = 0; i < kPrIntervals; ++i) slopes[i] = (values[i + 1] - values[i]) / (nodes[i + 1] - nodes[i]);
+    e = cudaMemcpyToSymbol(c_pr_nodes, nodes, sizeof nodes);
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(c_pr_values, values, sizeof values, sizeof(double) * (kPrIntervals + 1) * table);
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(c_pr_slopes, slopes, sizeof slopes, sizeof(double) * kPrIntervals * table);
+    if (e == cudaSuccess) done[dev][table] = true;
+    return e;
 }
 
 // ---- self test of the division shortcuts ------------------------------------------------------------

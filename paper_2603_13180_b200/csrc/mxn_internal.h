@@ -6,7 +6,7 @@
 
 namespace mxn {
 
-enum { STAT_NONE = 0, STAT_RMS = 1, STAT_MX = 2 };
+enum { STAT_NONE = 0, STAT_RMS = 1, STAT_MX = 2, STAT_POSTROUND = 3 };
 enum { ELEM_E4M3 = 0, ELEM_E2M1 = 1, ELEM_E5M2 = 2 };
 
 struct FwdParams {
@@ -23,6 +23,7 @@ struct FwdParams {
     int elem;               // ELEM_E4M3 (one byte per element) or ELEM_E2M1 (two elements per byte)
     // filled by the launcher
     int wpr, npass, rows_per_cta, tiles_per_row;
+    int pr_table;           // post-round estimator: index of the block size's f^-1 table
     double inv_count;       // 1/K (MXNorm) or 1/D (RMSNorm) when that is a power of two (exact), else 0
 };
 
@@ -30,6 +31,7 @@ bool fwd_shape_supported(int64_t D, int B);
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
 cudaError_t read_timeouts(unsigned int* out);
 cudaError_t selftest_division(unsigned long long* mismatches_host);
+cudaError_t postround_prepare(int B);   // uploads the f^-1 table for block size B to the current device (once)
 
 struct TransposedParams {
     const uint16_t* x;      // bf16 [T, D]

@@ -58,6 +58,8 @@ def run_fwd(binding, oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coe
     elif kind == "nvfp4":
         binding.mxnorm_nvfp4_fwd(x, codes, scales, rms, p=p, coef=coef, eps=eps, global_scale=global_scale,
                                  layout=layout)
+    elif kind == "postround":
+        binding.mxnorm_postround_fwd(x, codes, scales, rms, eps=eps, block=B, layout=layout)
     elif kind == "rms_nvfp4":
         binding.rmsnorm_nvfp4_fwd(x, codes, scales, rms, eps=eps, global_scale=global_scale, layout=layout)
     elif kind == "cast4":
@@ -93,6 +95,8 @@ def run_ref(oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coef=0.0, ep
         return oracle.mxnorm_ref(x_bits, gain=gain_bits, p=p, coef=coef, eps=eps, block=block, mode=round)
     if kind == "nvfp4":
         return oracle.mxnorm_nvfp4_ref(x_bits, p=p, coef=coef, eps=eps, global_scale=global_scale)
+    if kind == "postround":
+        return oracle.mxnorm_postround_ref(x_bits, eps=eps, block=block)
     if kind == "rms_nvfp4":
         return oracle.rmsnorm_nvfp4_ref(x_bits, eps=eps, global_scale=global_scale)
     if kind == "cast4":

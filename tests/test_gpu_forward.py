@@ -242,3 +242,24 @@ def test_rmsnorm_nvfp4_matches_oracle(binding, oracle, T, D):
 
 def test_division_shortcuts_equal_ieee_division(binding):
     assert binding.selftest_division() == 0
+
+
+@pytest.mark.parametrize("block", [16, 32, 64])
+@pytest.mark.parametrize("T,D", [(5, 64), (37, 768), (33, 4096), (9, 2560), (3, 16384), (257, 2048)])
+def test_postround_mxnorm_matches_oracle(binding, oracle, T, D, block):
+    """The paper's ablation: RMS from power-of-two-rounded absmaxes through the f^-1 table.  The library and the oracle
+    each build their own table, so r~ is compared to 1e-6 and scales/codes within the rounding of rho."""
+    x, _ = rows(T, D, seed=19 * T + D + block)
+    x[0] = 0                                                    # a zero row
+    for eps in (1e-5, 0.0):
+        got = gu.run_fwd(binding, oracle, "postround", x, block=block, eps=eps)
+        want = gu.run_ref(oracle, "postround", x, block=block, eps=eps)
+        nz = want[2] != 0
+        assert np.all(got[2][~nz] == 0)
+        sel = lambda t: tuple(a[nz] for a in t)
+        gu.assert_within_rounding_of_rho(sel(got), sel(want), block, f"postround B={block} {T}x{D}")
+        assert np.array_equal(got[0][~nz], want[0][~nz]) and np.array_equal(got[1][~nz], want[1][~nz])
+    got = gu.run_fwd(binding, oracle, "postround", x, block=block, eps=1e-5, layout=1)
+    want = gu.run_ref(oracle, "postround", x, block=block, eps=1e-5)
+    nz = want[2] != 0
+    gu.assert_within_rounding_of_rho(tuple(a[nz] for a in got), tuple(a[nz] for a in want), block, "postround tiled")

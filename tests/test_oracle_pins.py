@@ -499,6 +499,49 @@ def test_e5m2_element_format(oracle):
     assert np.array_equal(ct, c2) and np.array_equal(st, s2)
 
 
+def test_postround_estimator(oracle):
+    """Post-round MXNorm: f(sigma) = E[max_i 2^floor(log2 |X_i|)] against Monte Carlo, the scaling identity
+    f(2 sigma) = 2 f(sigma) the appendix states, f^-1 o f = id, and the estimator on Gaussian rows."""
+    rng = np.random.default_rng(0)
+    for B in (16, 32, 64):
+        for sigma in (1.0, 0.37, 5.3):
+            z = np.abs(rng.standard_normal((200000, B))) * sigma
+            mc = np.exp2(np.floor(np.log2(z.max(-1)))).mean()
+            f = oracle.postround_f(sigma, B)
+            assert abs(f - mc) < 4e-3 * mc, (B, sigma, f, mc)
+            assert abs(oracle.postround_f(2 * sigma, B) - 2 * f) < 1e-12 * f
+            assert abs(oracle.postround_f_inverse(f, B) - sigma) < 1e-12 * sigma
+        assert oracle.postround_f(1.0, B) < oracle.postround_f(1.01, B)          # increasing
+    # estimator: r~ tracks the RMS of Gaussian rows (it is noisier than the pre-round estimator)
+    x = wl.bits(wl.gaussian(512, 4096, seed=40, row_scale_sigma=1.0))
+    xv = bf16_vals(x).astype(np.float64)
+    rms = np.sqrt((xv ** 2).mean(-1))
+    for B in (16, 32):
+        codes, scales, r = oracle.mxnorm_postround_ref(x, block=B)
+        ratio = r / rms
+        assert abs(ratio.mean() - 1) < 0.01 and ratio.std() < 0.06, (B, ratio.mean(), ratio.std())
+        # r~ = f^-1(mean of rounded absmaxes), re-derived with exact bisection instead of the table: within the
+        # interpolation error of a 64-interval table
+        m = np.abs(xv).reshape(512, -1, B).max(-1)
+        xbar = np.exp2(np.floor(np.log2(m))).mean(-1)
+        for t in (0, 17, 511):
+            exact = oracle.postround_f_inverse(float(xbar[t]), B)
+            assert abs(r[t] - exact) < 2e-3 * exact
+        # scales and codes follow Algorithm 2 with this r~
+        rho = (np.float32(1.0) / r).astype(np.float32)
+        y = (bf16_vals(x) * rho[:, None]).astype(np.float32)
+        sb = smallest_pow2_scale(np.abs(y).reshape(512, -1, B).max(-1))
+        assert np.array_equal(scales, sb)
+    # 2^k shift: xbar scales exactly, the table is scale free -> r~ scales exactly, codes and scales unchanged
+    c0, s0, r0 = oracle.mxnorm_postround_ref(x[:32])
+    xs = bf16_bits(bf16_vals(x[:32]) * np.float32(2.0 ** -7))
+    c1, s1, r1 = oracle.mxnorm_postround_ref(xs)
+    assert np.array_equal(c0, c1) and np.array_equal(s0, s1) and np.array_equal(r1, r0 * np.float32(2.0 ** -7))
+    z = np.zeros((1, 64), np.uint16)
+    c, s_, r = oracle.mxnorm_postround_ref(z, eps=1e-5)
+    assert np.all(c == 0) and np.all(s_ == 0) and r[0] == 0
+
+
 # ------------------------------------------------------------------ library restatements
 def test_rms_estimate_against_numpy_restatement(oracle):
     x = _rand_rows(7, T=64, D=1024)
