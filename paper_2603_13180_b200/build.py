@@ -15,6 +15,7 @@ HEADERS = ["mxn_device.cuh", "mxn_internal.h", os.path.join("..", "..", "include
 # power-of-two products.
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "--ftz=false", "--prec-div=true", "--prec-sqrt=true",
+              "--split-compile", "0",   # the many template instantiations compile in parallel
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
 
 
@@ -27,16 +28,31 @@ def _stale() -> bool:
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compiles every translation unit in parallel (nvcc -c) and links libmxnorm.so next to this file."""
     if force or _stale():
-        tmp = LIB + f".tmp{os.getpid()}"
-        cmd = ["nvcc", *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp,
-               *[os.path.join(CSRC, f) for f in SOURCES]]
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        if verbose:
-            sys.stderr.write(res.stderr)
-        if res.returncode != 0:
-            raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-        os.replace(tmp, LIB)
+        import concurrent.futures
+        import tempfile
+        compile_flags = [f for f in NVCC_FLAGS if f not in ("-shared",)]
+        with tempfile.TemporaryDirectory(prefix="mxnorm_build_") as tmpdir:
+            def compile_one(src):
+                obj = os.path.join(tmpdir, src.replace(".cu", ".o"))
+                cmd = ["nvcc", "-c", *compile_flags, *(["-Xptxas", "-v"] if verbose else []), "-o", obj, os.path.join(CSRC, src)]
+                res = subprocess.run(cmd, capture_output=True, text=True)
+                return src, obj, res
+            with concurrent.futures.ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+                results = list(pool.map(compile_one, SOURCES))
+            for src, obj, res in results:
+                if verbose:
+                    sys.stderr.write(res.stderr)
+                if res.returncode != 0:
+                    raise RuntimeError(f"nvcc failed on {src}:\n" + res.stdout + res.stderr)
+            tmp = LIB + f".tmp{os.getpid()}"
+            link = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "shared", "-o", tmp,
+                    *[obj for _, obj, _ in results]]
+            res = subprocess.run(link, capture_output=True, text=True)
+            if res.returncode != 0:
+                raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
+            os.replace(tmp, LIB)
     return LIB
 
 
