@@ -1,16 +1,19 @@
-// Forward kernels: MXCast, fused RMSNorm+MXCast (Algorithm 1) and MXNorm (Algorithm 2) with
-// E4M3 codes / E8M0 scales, and the NVFP4 variant of MXNorm (E2M1 codes / E4M3 scales).
+// Forward kernels: MXCast, fused RMSNorm+MXCast (Algorithm 1), MXNorm (Algorithm 2) and its post-round
+// ablation with E4M3 codes / E8M0 scales; the MXFP4 (E2M1 / E8M0), NVFP4 (E2M1 / E4M3 scales) and
+// E5M2 variants.
 //
 // Work decomposition (memory-bound streaming map with one scalar reduction per row):
-//   * a row is handled by a "row group" of WPR warps (1 for D <= 4096 at B = 32) and stays in
-//     registers between the statistics phase and the quantise phase - every input byte is read
-//     from HBM exactly once, with 32-byte loads that bypass L1;
+//   * a row is handled by a "row group" of WPR warps (2 for D = 4096 at B = 32: at most 64 elements
+//     per lane) and stays in registers between the statistics phase and the quantise phase - every
+//     input byte is read from HBM exactly once, with 32-byte loads that bypass L1;
 //   * one lane owns one whole block per pass (B contiguous elements = 2B bytes), so the block
 //     absmax needs no cross-lane traffic, the scale is computed once per block, a warp writes
 //     32 consecutive scale bytes and 32*B consecutive code bytes per pass;
 //   * the only cross-lane step is the row statistic: K = D/B block values (MXNorm) instead of
 //     D squares (RMSNorm), reduced in binary64 by shuffles (and through shared memory when a row
-//     spans several warps).
+//     spans several warps);
+//   * short-lived CTAs (one per 1-4 rows), launched with programmatic stream serialisation: measured
+//     faster on B200 than resident CTAs, with or without TMA staging.
 #include <cmath>
 #include <mutex>
 
