@@ -129,6 +129,16 @@ mxn_status mxnorm_fwd(const void* x_bf16, const void* gain_bf16_or_null,
                       void* codes_u8, void* scales_u8, float* rms_est_out_or_null,
                       mxn_round round, mxn_scale_layout layout, void* cuda_stream);
 
+/* Residual add fused in front of MXNorm.  In a pre-norm transformer block the residual branch is added right
+ * before the norm (the paper's layer benchmark, appendix "Full Layer Benchmarks", notes that this add is fused
+ * with the norm).  h = bf16(x + residual) (binary32 sum, one round-to-nearest-even to bf16) is written to
+ * h_out_bf16 [T, D] - the new residual stream, which may alias x_bf16 or residual_bf16 exactly (in-place) -
+ * and MXNorm (mxnorm_fwd without gain, the paper's rounding rule) is applied to h without re-reading it.
+ * Pointers 32-byte aligned. */
+mxn_status mxnorm_add_fwd(const void* x_bf16, const void* residual_bf16, int64_t T, int64_t D, int block, int p,
+                          float coef_or_0, float eps, void* h_out_bf16, void* codes_u8, void* scales_u8,
+                          float* rms_est_out_or_null, mxn_scale_layout layout, void* cuda_stream);
+
 /* Post-round MXNorm - appendix "Post-round MXNorm" (the paper's ablation; it reports this variant unstable at
  * 8B parameters): the RMS is estimated from the block absmaxes after rounding them to powers of two,
  *   xbar = (1/K) sum_k 2^floor(log2 m_k),  r~ = f^-1(xbar),  f(sigma) = E[max_i 2^floor(log2 |X_i|)] for a block

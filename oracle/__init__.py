@@ -54,6 +54,8 @@ def _load():
         lib.rmsnorm_nvfp4_ref.restype = i32
         lib.mxnorm_postround_ref.argtypes = [vp, i64, i64, i32, f32, i32, vp, vp, vp]
         lib.mxnorm_postround_ref.restype = i32
+        lib.mxnorm_add_ref.argtypes = [vp, vp, i64, i64, i32, i32, f32, f32, i32, vp, vp, vp, vp]
+        lib.mxnorm_add_ref.restype = i32
         lib.mxn_ref_postround_f.argtypes = [ctypes.c_double, i32]
         lib.mxn_ref_postround_f.restype = ctypes.c_double
         lib.mxn_ref_postround_f_inverse.argtypes = [ctypes.c_double, i32]
@@ -173,6 +175,21 @@ def rmsnorm_nvfp4_ref(x, eps=0.0, global_scale=1.0):
     _check(_load().rmsnorm_nvfp4_ref(_p(x), T, D, eps, global_scale, _p(codes), _p(scales), _p(rms)),
            "rmsnorm_nvfp4_ref")
     return codes, scales, rms
+
+
+def mxnorm_add_ref(x, res, p=2, coef=0.0, eps=0.0, block=32, mode=ROUND_RCEIL_POW2):
+    """Residual add then MXNorm: returns (h [T, D] bf16 bits, codes, scales, rms_estimate)."""
+    x = _bf16(x, 2)
+    res = _bf16(res, 2)
+    assert x.shape == res.shape
+    T, D = x.shape
+    h = np.zeros((T, D), np.uint16)
+    codes = np.zeros((T, D), np.uint8)
+    scales = np.zeros((T, D // block if D % block == 0 else 0), np.uint8)
+    rms = np.zeros((T,), np.float32)
+    _check(_load().mxnorm_add_ref(_p(x), _p(res), T, D, block, p, coef, eps, mode, _p(h), _p(codes), _p(scales), _p(rms)),
+           "mxnorm_add_ref")
+    return h, codes, scales, rms
 
 
 def mxnorm_postround_ref(x, eps=0.0, block=32, mode=ROUND_RCEIL_POW2):

@@ -499,6 +499,31 @@ int mxnorm_bwd_ref(const uint16_t *x_bf16, const uint16_t *g_bf16, const uint16_
 }
 
 /* ------------------------------------------------------------------------- */
+/* O8  Residual add fused in front of MXNorm (pre-norm transformer blocks add  */
+/*     the residual branch right before the norm; the layer benchmark of the   */
+/*     paper notes that this add is fused with the norm).                      */
+/*     h = bf16(fl32(x) + fl32(res)) (round-to-nearest-even to bf16), written  */
+/*     out as the new residual stream; then Algorithm 2 on h.                  */
+/* ------------------------------------------------------------------------- */
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040); /* NaN stays NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+int mxnorm_add_ref(const uint16_t *x_bf16, const uint16_t *res_bf16, int64_t T, int64_t D, int B, int p, float coef,
+                   float eps, int mode, uint16_t *h_bf16, uint8_t *codes, uint8_t *scales, float *rms_est_out)
+{
+    if (!shape_ok(T, D, B) || (p != 1 && p != 2)) return 1;
+    for (int64_t i = 0; i < T * D; ++i) h_bf16[i] = f32_to_bf16_rne(bf16_to_f32(x_bf16[i]) + bf16_to_f32(res_bf16[i]));
+    return mxnorm_ref(h_bf16, NULL, T, D, B, p, coef, eps, mode, REF_ELEM_E4M3, codes, scales, rms_est_out);
+}
+
+/* ------------------------------------------------------------------------- */
 /* O7  Post-round MXNorm (appendix "Post-round MXNorm"): the RMS is estimated    */
 /*     from the block absmaxes AFTER rounding them to powers of two,            */
 /*       s_k = r(m_k) = 2^floor(log2 m_k)   (0 for a zero block),                */

@@ -23,7 +23,8 @@ EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
            "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
-           "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd")
+           "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
+           "mxnorm_add_fwd")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -54,6 +55,7 @@ lib.mxnorm_fwd_host_workspace_bytes.restype = _sz
 lib.mx_cast_fp4.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.rmsnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mxnorm_mxfp4_fwd.argtypes = [_vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.mxnorm_add_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _vp, _i32, _vp]
 lib.mxnorm_postround_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _vp]
 lib.mx_cast_e5m2.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.mx_cast_transposed_e5m2.argtypes = [_vp, _i64, _i64, _vp, _vp, _i32, _vp]
@@ -65,7 +67,8 @@ lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
 for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
               "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
-           "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd"):
+           "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
+           "mxnorm_add_fwd"):
     getattr(lib, _name).restype = _i32
 
 
@@ -260,3 +263,13 @@ def mxnorm_postround_fwd(x, codes, scales, rms_est_out=None, eps=0.0, block=32, 
     T, D = x.shape
     _check(lib.mxnorm_postround_fwd(_ptr(x), T, D, block, eps, _ptr(codes), _ptr(scales), _ptr(rms_est_out), layout,
                                     _stream(stream)), "mxnorm_postround_fwd")
+
+
+def mxnorm_add_fwd(x, residual, h_out, codes, scales, rms_est_out=None, p=2, coef=0.0, eps=0.0, block=32,
+                   layout=SCALES_ROWMAJOR, stream=None):
+    """h_out = bf16(x + residual) and MXNorm(h_out) in one pass (h_out may be x or residual itself)."""
+    _dev(x, torch.bfloat16, "x")
+    _dev(residual, torch.bfloat16, "residual")
+    T, D = x.shape
+    _check(lib.mxnorm_add_fwd(_ptr(x), _ptr(residual), T, D, block, p, coef, eps, _ptr(h_out), _ptr(codes), _ptr(scales),
+                              _ptr(rms_est_out), layout, _stream(stream)), "mxnorm_add_fwd")

@@ -161,6 +161,38 @@ mxn_status rmsnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, float eps
                    scales_e4m3, rms_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
 }
 
+mxn_status mxnorm_add_fwd(const void* x_bf16, const void* residual_bf16, int64_t T, int64_t D, int block, int p,
+                          float coef_or_0, float eps, void* h_out_bf16, void* codes_u8, void* scales_u8,
+                          float* rms_est_out_or_null, mxn_scale_layout layout, void* cuda_stream)
+{
+    mxn_status st = check_common(x_bf16, T, D, block, codes_u8, scales_u8, MXN_ROUND_RCEIL_POW2, layout);
+    if (st != MXN_OK || T == 0) return st;
+    if (residual_bf16 == nullptr || h_out_bf16 == nullptr) return MXN_ERR_NULL;
+    if (misaligned(residual_bf16, 32) || misaligned(h_out_bf16, 32)) return MXN_ERR_ALIGN;
+    if (p != 1 && p != 2) return MXN_ERR_SHAPE;
+    if (rms_est_out_or_null != nullptr && misaligned(rms_est_out_or_null, 4)) return MXN_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    mxn::FwdParams P{};
+    P.x = static_cast<const uint16_t*>(x_bf16);
+    P.residual = static_cast<const uint16_t*>(residual_bf16);
+    P.h_out = static_cast<uint16_t*>(h_out_bf16);
+    P.codes = static_cast<uint8_t*>(codes_u8);
+    P.scales = static_cast<uint8_t*>(scales_u8);
+    P.rms_out = rms_est_out_or_null;
+    P.T = T;
+    P.D = (int)D;
+    P.K = (int)(D / block);
+    P.p = p;
+    P.coef = coef_or_0 == 0.0f ? paper_coef(block, p) : coef_or_0;
+    P.eps = eps;
+    P.global_scale = 1.0f;
+    P.round = MXN_ROUND_RCEIL_POW2;
+    P.layout = layout;
+    P.elem = mxn::ELEM_E4M3;
+    if (clear_scale_padding(scales_u8, T, P.K, layout, s) != cudaSuccess) return MXN_ERR_CUDA;
+    return mxn::launch_fwd(P, block, mxn::STAT_MX, false, s) == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
+}
+
 mxn_status mxnorm_postround_fwd(const void* x_bf16, int64_t T, int64_t D, int block, float eps, void* codes_u8,
                                 void* scales_u8, float* rms_est_out_or_null, mxn_scale_layout layout, void* cuda_stream)
 {

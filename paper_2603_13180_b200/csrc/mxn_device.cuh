@@ -22,6 +22,13 @@ __device__ __forceinline__ void ld_v8(const void* p, uint32_t* r)
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "l"(p));
 }
+// same width through the coherent path: for buffers the kernel may also write (in-place residual update)
+__device__ __forceinline__ void ld_v8_coherent(const void* p, uint32_t* r)
+{
+    asm volatile("ld.global.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(p) : "memory");
+}
 __device__ __forceinline__ void st_v8(void* p, const uint32_t* r)
 {
     asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"

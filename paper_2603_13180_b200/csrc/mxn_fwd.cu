@@ -359,7 +359,7 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
 
 // ---- register-direct kernels: one row per row group, loaded straight from global memory -----------
 // Generic path: any D % B == 0, rows spanning up to 8 warps, optional gain.
-template <int B, int NPASS>
+template <int B, int NPASS, bool COHERENT = false>
 __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], const uint16_t* xrow, int K, int wpr, int w, int lane)
 {
     constexpr int W = B / 2;
@@ -369,7 +369,10 @@ __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], co
         if (k < K) {
             const uint16_t* p = xrow + (int64_t)k * B;
 #pragma unroll
-            for (int v = 0; v < W / 8; ++v) ld_v8(p + v * 16, &xr[i][v * 8]);
+            for (int v = 0; v < W / 8; ++v) {
+                if (COHERENT) ld_v8_coherent(p + v * 16, &xr[i][v * 8]);
+                else ld_v8(p + v * 16, &xr[i][v * 8]);
+            }
         } else {
 #pragma unroll
             for (int j = 0; j < W; ++j) xr[i][j] = 0u;
@@ -399,6 +402,54 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m
         if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     }
     quantise_store_e4m3<B, NPASS, WPR, GAIN, PAPER>(xr, m, rho, P, row, w, lane);
+}
+
+// Residual add fused in front of MXNorm: h = bf16(x + res) is written out as the new residual stream and
+// normalised from registers (reads 4D bytes, writes 2D + D + D/B per row instead of two passes over h).
+__device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b)
+{
+    // each half: binary32 sum of two exactly widened bf16 values, rounded once to bf16 (RN-even)
+    const float lo = __fadd_rn(bf16_lo(a), bf16_lo(b)), hi = __fadd_rn(bf16_hi(a), bf16_hi(b));
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+template <int B, int NPASS, int WPR>
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_add_mx_kernel(const FwdParams P)
+{
+    constexpr int W = B / 2;
+    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / WPR, w = warp - group * WPR;
+    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    pdl_prologue();
+    if (row >= P.T) return;
+
+    uint32_t xr[NPASS][W];
+    float m[NPASS];
+    load_row_direct<B, NPASS, true>(xr, P.x + row * P.D, P.K, WPR, w, lane);   // h_out may alias x or residual
+    {
+        uint32_t rr[NPASS][W];
+        load_row_direct<B, NPASS, true>(rr, P.residual + row * P.D, P.K, WPR, w, lane);
+        uint16_t* hrow = P.h_out + row * P.D;
+#pragma unroll
+        for (int i = 0; i < NPASS; ++i) {
+#pragma unroll
+            for (int j = 0; j < W; ++j) xr[i][j] = add_bf16x2(xr[i][j], rr[i][j]);
+            const int k = (i * WPR + w) * kWarp + lane;
+            if (k < P.K) {
+#pragma unroll
+                for (int v = 0; v < W / 8; ++v) st_v8(hrow + (int64_t)k * B + v * 16, &xr[i][v * 8]);
+            }
+        }
+    }
+    double stat = block_stats<B, NPASS, STAT_MX>(xr, m, P.p);
+    stat = group_sum<WPR>(stat, group, w, red);
+    float r, rho;
+    finish_stat<STAT_MX>(stat, P, r, rho);
+    if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    quantise_store_e4m3<B, NPASS, WPR, false, true>(xr, m, rho, P, row, w, lane);
 }
 
 // plain MXCast to E5M2 codes (gradient tensors), the paper's rounding rule with 2^15
@@ -548,6 +599,23 @@ static fwd_fn pick_mxfp4(int wpr, int npass)
     }
 }
 template <int B>
+static fwd_fn pick_add_mx(int wpr, int npass)
+{
+    constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
+    if (wpr == 2) return fwd_add_mx_kernel<B, MAXP, 2>;
+    if (wpr == 4) return fwd_add_mx_kernel<B, MAXP, 4>;
+    if (wpr == 8) return fwd_add_mx_kernel<B, MAXP, 8>;
+    if (wpr == 16) return fwd_add_mx_kernel<B, MAXP, 16>;
+    if (wpr != 1) return nullptr;
+    switch (npass) {
+        case 1: return fwd_add_mx_kernel<B, 1, 1>;
+        case 2: return fwd_add_mx_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1>;
+        case 3: return fwd_add_mx_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1>;
+        default: return fwd_add_mx_kernel<B, MAXP, 1>;
+    }
+}
+
+template <int B>
 static fwd_fn pick_e5m2(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
@@ -641,7 +709,8 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
 {
     const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
     const bool e5m2 = P.elem == ELEM_E5M2;
-    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && stat != STAT_POSTROUND && B == 32 && P.gain == nullptr &&
+    const bool add = P.residual != nullptr;
+    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && !add && stat != STAT_POSTROUND && B == 32 && P.gain == nullptr &&
                                 P.round == MXN_ROUND_RCEIL_POW2);
     P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
     if (!plan_row(P.K, B, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
@@ -654,6 +723,7 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
     if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
+    else if (add) fn = B == 16 ? pick_add_mx<16>(P.wpr, P.npass) : B == 32 ? pick_add_mx<32>(P.wpr, P.npass) : pick_add_mx<64>(P.wpr, P.npass);
     else if (e5m2) fn = B == 16 ? pick_e5m2<16>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32>(P.wpr, P.npass) : pick_e5m2<64>(P.wpr, P.npass);
     else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16>(stat, P.wpr, P.npass)
                        : B == 32 ? pick_mxfp4_stat<32>(stat, P.wpr, P.npass) : pick_mxfp4_stat<64>(stat, P.wpr, P.npass);

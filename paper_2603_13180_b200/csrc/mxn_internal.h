@@ -12,6 +12,8 @@ enum { ELEM_E4M3 = 0, ELEM_E2M1 = 1, ELEM_E5M2 = 2 };
 struct FwdParams {
     const uint16_t* x;      // bf16 [T, D]
     const uint16_t* gain;   // bf16 [D] or nullptr
+    const uint16_t* residual; // bf16 [T, D] or nullptr: added to x before the norm (fused residual add)
+    uint16_t* h_out;        // bf16 [T, D]: x + residual, written when residual is given
     uint8_t* codes;         // [T, D] (E4M3) or [T, D/2] (E2M1 pairs)
     uint8_t* scales;        // row-major [T, K] or 128x4-tiled
     float* rms_out;         // [T] or nullptr
@@ -51,6 +53,8 @@ struct BwdParams {
     const uint16_t* x;      // bf16 [T, D]
     const uint16_t* g;      // bf16 [T, D]
     const uint16_t* gain;   // bf16 [D] or nullptr
+    const uint16_t* residual; // bf16 [T, D] or nullptr: added to x before the norm (fused residual add)
+    uint16_t* h_out;        // bf16 [T, D]: x + residual, written when residual is given
     const float* rms;       // [T]
     void* dx;               // bf16 or fp32 [T, D]
     float* dgain;           // [D] or nullptr

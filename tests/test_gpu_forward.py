@@ -263,3 +263,25 @@ def test_postround_mxnorm_matches_oracle(binding, oracle, T, D, block):
     want = gu.run_ref(oracle, "postround", x, block=block, eps=1e-5)
     nz = want[2] != 0
     gu.assert_within_rounding_of_rho(tuple(a[nz] for a in got), tuple(a[nz] for a in want), block, "postround tiled")
+
+
+@pytest.mark.parametrize("block", [16, 32, 64])
+@pytest.mark.parametrize("T,D", [(5, 64), (37, 768), (33, 4096), (9, 2560), (3, 16384), (257, 2048)])
+def test_residual_add_then_mxnorm_matches_oracle(binding, oracle, T, D, block):
+    x, _ = rows(T, D, seed=23 * T + D + block)
+    res, _ = rows(T, D, seed=29 * T + D + block)
+    res[0] = x[0] ^ 0x8000                                      # exact cancellation: a zero row
+    want_h, wc, ws, wr = oracle.mxnorm_add_ref(x, res, eps=1e-5, block=block)
+    xg, rg = wl.from_bits(x).cuda(), wl.from_bits(res).cuda()
+    for inplace in (False, True):
+        hfull, hbytes = gu.guarded(T * D * 2)
+        h = hbytes.view(torch.bfloat16).view(T, D)
+        codes, scales, rms = binding.alloc_outputs(T, D, block)
+        target = xg.clone() if inplace else h
+        binding.mxnorm_add_fwd(target if inplace else xg, rg, target, codes, scales, rms, eps=1e-5, block=block)
+        torch.cuda.synchronize()
+        assert gu.guards_intact(hfull, T * D * 2)
+        assert np.array_equal(wl.bits(target.cpu()), want_h)
+        assert np.array_equal(codes.cpu().numpy(), wc)
+        assert np.array_equal(scales.cpu().numpy().reshape(T, D // block), ws)
+        assert np.array_equal(rms.cpu().numpy(), wr)

@@ -542,6 +542,19 @@ def test_postround_estimator(oracle):
     assert np.all(c == 0) and np.all(s_ == 0) and r[0] == 0
 
 
+def test_residual_add_then_mxnorm(oracle):
+    """h = bf16(x + res) must be torch's bf16 addition bit for bit, and the rest is Algorithm 2 on h."""
+    a = wl.make_inputs(wl.Workload("t", 40, 512, seed=50, outlier_frac=0.004))["x"]
+    b = wl.make_inputs(wl.Workload("t", 40, 512, seed=51))["x"] * 3
+    b[3] = -a[3]                                              # exact cancellation -> a zero row
+    b[4, ::2] = a[4, ::2] * 2.0 ** -12                          # tiny addends: rounding of the sum matters
+    h, codes, scales, r = oracle.mxnorm_add_ref(wl.bits(a), wl.bits(b), eps=1e-5)
+    assert np.array_equal(h, wl.bits(a + b))                  # torch adds bf16 tensors in fp32 and rounds once (RN-even)
+    c2, s2, r2 = oracle.mxnorm_ref(h, eps=1e-5)
+    assert np.array_equal(codes, c2) and np.array_equal(scales, s2) and np.array_equal(r, r2)
+    assert r[3] == 0 and np.all(codes[3] & 0x7F == 0)
+
+
 # ------------------------------------------------------------------ library restatements
 def test_rms_estimate_against_numpy_restatement(oracle):
     x = _rand_rows(7, T=64, D=1024)
