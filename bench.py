@@ -184,6 +184,9 @@ def profile_run(mx, xs, outs, T, D, layout, fwd, rms, cast):
         mx.mxnorm_mxfp4_fwd(xs[i], m4[0], m4[1], m4[2], eps=EPS, layout=layout)
         mx.mxnorm_bwd(xs[i], g, gain, r, dx, dgain, ws)
         mx.mx_cast_transposed(xs[i], r, ct, st, eps=EPS, layout=layout)
+        mx.rmsnorm_nvfp4_fwd(xs[i], o4[0], o4[1], o4[2], eps=EPS)
+        mx.mxnorm_postround_fwd(xs[i], c, s, r, eps=EPS, layout=layout)
+        mx.mxnorm_add_fwd(xs[i], xs[(i + 1) % len(xs)], dx, c, s, r, eps=EPS, layout=layout)
     torch.cuda.synchronize()
     print(json.dumps({"profile_run": "3 launches of each kernel", "rows": T, "hidden": D, "timeouts": mx.device_timeouts()}))
 
@@ -399,6 +402,27 @@ def main():
             mst = time_launches(transposed, SETS, args.steps, args.warmup, stream)
             others["mx_cast_transposed"] = {"ms": mst, "gbs": (T * D * 3 + T * D // 32 + 4 * T) / mst / 1e6}
             del ct, stt
+        # the ablation with power-of-two-rounded block maxima, and the residual add fused in front
+        def postround(i):
+            c, s, r = outs[i]
+            st = L.mxnorm_postround_fwd(xs[i].data_ptr(), T, D, 32, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(), layout, sh)
+            if st != 0:
+                raise RuntimeError(mx.status_string(st))
+
+        mspr = time_launches(postround, SETS, args.steps, args.warmup, stream)
+        others["mxnorm_postround_fwd"] = {"ms": mspr, "gbs": algorithmic_bytes("mx", T, D) / mspr / 1e6}
+        hs = [torch.empty_like(xs[0]) for _ in range(SETS)]
+
+        def add_fwd(i):
+            c, s, r = outs[i]
+            st = L.mxnorm_add_fwd(xs[i].data_ptr(), xs[(i + 1) % SETS].data_ptr(), T, D, 32, 2, 0.0, EPS, hs[i].data_ptr(),
+                                  c.data_ptr(), s.data_ptr(), r.data_ptr(), layout, sh)
+            if st != 0:
+                raise RuntimeError(mx.status_string(st))
+
+        msadd = time_launches(add_fwd, SETS, args.steps, args.warmup, stream)
+        others["mxnorm_add_fwd"] = {"ms": msadd, "gbs": (algorithmic_bytes("mx", T, D) + 4 * T * D) / msadd / 1e6}
+        del hs
         # backward (C5 tensors: seed 1, gradient ~ N(0, 1e-2), gain)
         w5 = wl.CONFIGS["C5"]
         inp5 = wl.make_inputs(w5) if T == w5.T else wl.make_inputs(w5, T=T)
