@@ -33,6 +33,11 @@
  *    libmxnorm kernel and is itself launched with the programmatic attribute must do the same wait
  *    (griddepcontrol.wait / cudaGridDependencySynchronize) before reading libmxnorm's outputs;
  *    ordinary launches need nothing.
+ *  - Stream capture: every device-pointer entry point only enqueues kernels (and, for a tiled scale
+ *    buffer with padding, one memset) on `cuda_stream`, so it may be called while that stream is being
+ *    captured into a CUDA graph; the exceptions are stated at the entry points concerned (the first
+ *    call of mxnorm_postround_fwd per block size and the first call of mxnorm_bwd_noalloc and of
+ *    mxnorm_fwd_host per device do one-time set-up that is not capturable).
  *  - Outputs are fully overwritten.  Inputs must be finite; results for NaN/Inf
  *    inputs are unspecified (no fault).
  *  - Every function returns a status; nothing aborts, throws or prints.  Argument
