@@ -326,6 +326,9 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
 {
     const float rho_g = __fmul_rn(rho, P.global_scale);
     const bool rho_g_in_window = in_division_window(rho_g);
+    // RN(1/(1+j/8)), j = lane % 8, held one per lane and fetched with a shuffle: a lane-dependent index into
+    // constant memory would be replayed once per distinct index
+    const float rcp_sig = kRcpE4M3Significand[lane & 7];
     uint8_t* cp0 = P.codes + row * (P.D / 2) + (int64_t)(w * kWarp + lane) * 8;
     int64_t soff, sstep;
     scale_addressing<WPR>(P, row, w, lane, soff, sstep);
@@ -333,14 +336,24 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
         const int k = (i * WPR + w) * kWarp + lane;
-        // block scale = E4M3(fl32(fl32(a/6) * global_scale)), a = fl32(m * rho~)
+        // block scale = E4M3(fl32(fl32(a/6) * global_scale)), a = fl32(m * rho~);
+        // element factor = fl32(rho~ * global_scale) / scale (0 when the scale is 0)
         const float a = __fmul_rn(m[i], rho);
-        const float t = __fmul_rn(div_by_6(a), P.global_scale);
-        const uint32_t sc = cvt_e4m3x2(t, 0.0f) & 0xFFu;
-        const float d = e4m3_to_f32(sc);
+        // the common case first, without the IEEE division sequences and decided for the whole warp at once:
+        // numerators inside the window of the exact shortcut and a normal E4M3 scale
+        uint32_t sc = cvt_e4m3x2(__fmul_rn(div_by_known(a, 6.0f, 0x1.555556p-3f), P.global_scale), 0.0f) & 0xFFu;
+        const bool common = in_division_window(a) && sc >= 8u && rho_g_in_window;
         float inv;
-        if (sc >= 8u && rho_g_in_window) inv = div_by_e4m3_normal(rho_g, sc, d);   // normal scale: no division sequence
-        else inv = d == 0.0f ? 0.0f : __fdiv_rn(rho_g, d);
+        if (__all_sync(0xFFFFFFFFu, common || k >= P.K)) {
+            const float d = __uint_as_float((sc << 20) + (120u << 23));            // (8+mf) * 2^(ef-10)
+            const float c = __fmul_rn(__shfl_sync(0xFFFFFFFFu, rcp_sig, (int)(sc & 7u)), __uint_as_float((134u - (sc >> 3)) << 23));
+            inv = div_by_known(rho_g, d, c);
+        } else {
+            sc = cvt_e4m3x2(__fmul_rn(div_by_6(a), P.global_scale), 0.0f) & 0xFFu;
+            const float d = e4m3_to_f32(sc);
+            if (sc >= 8u && rho_g_in_window) inv = div_by_e4m3_normal(rho_g, sc, d);
+            else inv = d == 0.0f ? 0.0f : __fdiv_rn(rho_g, d);
+        }
         uint32_t out[2];
         const float2 ii = make_float2(inv, inv);
 #pragma unroll
