@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
     }
 
     uint32_t gam[V][4];   // gain kept as packed bf16 pairs
-    float acc[V][8];
+    float2 acc[V][4];
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int vi = tid + v * n;
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
         if (GAIN && vi < nvec) gw = __ldg(reinterpret_cast<const uint4*>(P.gain) + vi);
         gam[v][0] = gw.x; gam[v][1] = gw.y; gam[v][2] = gw.z; gam[v][3] = gw.w;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[v][j] = 0.0f;
+        for (int j = 0; j < 4; ++j) acc[v][j] = make_float2(0.0f, 0.0f);
     }
     __syncthreads();   // barriers initialised before anyone waits on them
 
@@ -150,27 +150,26 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
 
         // One pass over the thread's elements with  gi = g/r,  t = gi*gamma (= h/r):
         //   dgamma += x*gi ;  dot += t*x  (= sum_d h x / r) ;  later  dX = t - x * (dot/(D r^2)).
-        float tt[V][8];
-        float d0 = 0.f, d1 = 0.f;
+        // (two elements per instruction: packed binary32 multiply and fused multiply-add, each half an
+        //  ordinary IEEE operation)
+        float2 tt[V][4];
+        float2 dd = make_float2(0.f, 0.f);
+        const float2 inv_r2 = make_float2(inv_r, inv_r);
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
             const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float x0 = bf16_lo(xa[j]), x1 = bf16_hi(xa[j]);
-                const float gi0 = bf16_lo(ga[j]) * inv_r, gi1 = bf16_hi(ga[j]) * inv_r;
-                if (DGAIN) {
-                    acc[v][2 * j] = fmaf(x0, gi0, acc[v][2 * j]);
-                    acc[v][2 * j + 1] = fmaf(x1, gi1, acc[v][2 * j + 1]);
-                }
-                const float t0 = GAIN ? gi0 * bf16_lo(gam[v][j]) : gi0, t1 = GAIN ? gi1 * bf16_hi(gam[v][j]) : gi1;
-                tt[v][2 * j] = t0;
-                tt[v][2 * j + 1] = t1;
-                d0 = fmaf(t0, x0, d0);
-                d1 = fmaf(t1, x1, d1);
+                const float2 x2 = bf16x2_to_f32x2(xa[j]);
+                const float2 gi = mul2(bf16x2_to_f32x2(ga[j]), inv_r2);
+                if (DGAIN) acc[v][j] = __ffma2_rn(x2, gi, acc[v][j]);
+                const float2 t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gam[v][j])) : gi;
+                tt[v][j] = t2;
+                dd = __ffma2_rn(t2, x2, dd);
             }
         }
+        const float d0 = dd.x, d1 = dd.y;
         const float dot = warp_sum(d0 + d1);
         if (lane == 0) red[it & 1][warp] = dot;
         __syncthreads();   // row dot complete; every thread has read its part of the stage
@@ -195,20 +194,18 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
             const int vi = tid + v * n;
             if (vi >= nvec) continue;
             const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
-            float o[8];
+            float2 o[4];
+            const float2 nc2 = make_float2(-c2, -c2);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                o[2 * j] = fmaf(-bf16_lo(xa[j]), c2, tt[v][2 * j]);
-                o[2 * j + 1] = fmaf(-bf16_hi(xa[j]), c2, tt[v][2 * j + 1]);
-            }
+            for (int j = 0; j < 4; ++j) o[j] = __ffma2_rn(bf16x2_to_f32x2(xa[j]), nc2, tt[v][j]);
             if (P.dx_is_fp32) {
                 float* dp = static_cast<float*>(P.dx) + row * P.D + (int64_t)vi * 8;
-                st_v4(dp, reinterpret_cast<const uint32_t*>(o));
-                st_v4(dp + 4, reinterpret_cast<const uint32_t*>(o + 4));
+                st_v4(dp, reinterpret_cast<const uint32_t*>(&o[0]));
+                st_v4(dp + 4, reinterpret_cast<const uint32_t*>(&o[2]));
             } else {
                 uint32_t pk[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) pk[j] = pack_bf16x2(o[2 * j], o[2 * j + 1]);
+                for (int j = 0; j < 4; ++j) pk[j] = pack_bf16x2(o[j].x, o[j].y);
                 st_v4(static_cast<uint16_t*>(P.dx) + row * P.D + (int64_t)vi * 8, pk);
             }
         }
@@ -221,8 +218,8 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
             const int vi = tid + v * n;
             if (vi < nvec) {
                 float4* q = reinterpret_cast<float4*>(prow + (int64_t)vi * 8);
-                q[0] = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
-                q[1] = make_float4(acc[v][4], acc[v][5], acc[v][6], acc[v][7]);
+                q[0] = make_float4(acc[v][0].x, acc[v][0].y, acc[v][1].x, acc[v][1].y);
+                q[1] = make_float4(acc[v][2].x, acc[v][2].y, acc[v][3].x, acc[v][3].y);
             }
         }
     }
