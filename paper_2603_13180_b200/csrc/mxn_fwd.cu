@@ -8,7 +8,9 @@
 //     input byte is read from HBM exactly once, with 32-byte loads that bypass L1;
 //   * one lane owns one whole block per pass (B contiguous elements = 2B bytes), so the block
 //     absmax needs no cross-lane traffic, the scale is computed once per block, a warp writes
-//     32 consecutive scale bytes and 32*B consecutive code bytes per pass;
+//     32 consecutive scale bytes and 32*B consecutive code bytes per pass (B = 64: two adjacent lanes
+//     own the halves of a block - LPB = 2 "lanes per block" - and exchange their maxima with one shuffle,
+//     which keeps a lane at 32 contiguous elements per pass and the per-lane code identical to B = 32);
 //   * the only cross-lane step is the row statistic: K = D/B block values (MXNorm) instead of
 //     D squares (RMSNorm), reduced in binary64 by shuffles (and through shared memory when a row
 //     spans several warps);
@@ -116,12 +118,13 @@ __device__ __forceinline__ double group_sum(double v, int group, int w, double* 
 }
 
 // ---- per-row work -------------------------------------------------------------------------------
-// Lane `lane` of pass i of warp w owns block k = (i*wpr + w)*32 + lane; xr[i][] holds its B bf16
-// values as packed pairs (zeros when k >= K).
+// Lane `lane` of pass i of warp w owns piece k = (i*wpr + w)*32 + lane of the row: B contiguous elements,
+// held in xr[i][] as packed pairs (zeros when k >= P.chunks).  A block of the format is LPB adjacent
+// pieces (LPB = 1: the piece is the block).
 
 // phase 1: block absmaxes m[i] (exact) and this lane's share of the row statistic
-template <int B, int NPASS, int STAT>
-__device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2], float (&m)[NPASS], int p)
+template <int B, int NPASS, int STAT, int LPB = 1>
+__device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2], float (&m)[NPASS], int p, int lane = 0)
 {
     constexpr int W = B / 2;
     double stat = 0.0;
@@ -132,12 +135,15 @@ __device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2]
 #pragma unroll
         for (int j = 2; j < W; ++j) m2 = absmax_bf16x2(m2, xr[i][j]);
         m[i] = hmax_abs_to_f32(m2);
+#pragma unroll
+        for (int o = 1; o < LPB; o <<= 1) m[i] = fmaxf(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], o));   // block absmax in every lane of the block
+        const float mc = (LPB == 1 || (lane & (LPB - 1)) == 0) ? m[i] : 0.0f;   // each block counted once (adding 0 is exact)
         if (STAT == STAT_MX) {
-            double md = (double)m[i];
+            double md = (double)mc;
             stat = p == 2 ? __fma_rn(md, md, stat) : __dadd_rn(stat, md);   // m^2 is exact in binary64
         }
         if (STAT == STAT_POSTROUND)   // 2^floor(log2 m): the absmax with its significand cleared (0 stays 0)
-            stat = __dadd_rn(stat, (double)__uint_as_float(__float_as_uint(m[i]) & 0x7F800000u));
+            stat = __dadd_rn(stat, (double)__uint_as_float(__float_as_uint(mc) & 0x7F800000u));
         if (STAT == STAT_RMS) {
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
@@ -162,24 +168,25 @@ __device__ __forceinline__ void forget_unpacked(uint32_t (&xr)[NPASS][W])
         for (int j = 0; j < W; ++j) asm volatile("" : "+r"(xr[i][j]));
 }
 
-// byte offset of this lane's first scale (pass 0) and the distance between passes
-template <int WPR>
+// byte offset of the scale of this lane's first block (pass 0) and the distance between passes
+template <int WPR, int LPB = 1>
 __device__ __forceinline__ void scale_addressing(const FwdParams& P, int64_t row, int w, int lane, int64_t& off0, int64_t& step)
 {
-    const int k0 = w * kWarp + lane;
+    static_assert((kWarp / LPB) % 4 == 0, "a pass of one warp must cover whole groups of four scales");
+    const int k0 = (w * kWarp + lane) / LPB;
     if (P.layout == MXN_SCALES_ROWMAJOR) {
         off0 = row * P.K + k0;
-        step = WPR * kWarp;
+        step = WPR * (kWarp / LPB);
     } else {
         const int rr = (int)(row & 127);
         off0 = ((row >> 7) * P.tiles_per_row + (k0 >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (k0 & 3);
-        step = (int64_t)WPR * (kWarp / 4) * 512;   // 32*WPR blocks further = 8*WPR tiles of 512 bytes
+        step = (int64_t)WPR * (kWarp / LPB / 4) * 512;   // 32*WPR/LPB blocks further = that many / 4 tiles of 512 bytes
     }
 }
 
 // phase 2 (E4M3 codes, E8M0 scales): scales, codes and their stores for this lane's blocks.
 // PAPER selects the paper's rounding rule at compile time (the common case); otherwise P.round decides.
-template <int B, int NPASS, int WPR, bool GAIN, bool PAPER, int ELEM = 0>
+template <int B, int NPASS, int WPR, bool GAIN, bool PAPER, int ELEM = 0, int LPB = 1>
 __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][B / 2], const float (&m)[NPASS], float rho,
                                                     const FwdParams& P, int64_t row, int w, int lane)
 {
@@ -187,12 +194,12 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
     const bool rho_normal = is_normal_f32(rho);
     uint8_t* cp0 = P.codes + row * P.D + (int64_t)(w * kWarp + lane) * B;
     int64_t soff, sstep;
-    scale_addressing<WPR>(P, row, w, lane, soff, sstep);
+    scale_addressing<WPR, LPB>(P, row, w, lane, soff, sstep);
     uint8_t* sp0 = P.scales + soff;
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
         const int k = (i * WPR + w) * kWarp + lane;
-        const bool active = k < P.K;
+        const bool active = k < P.chunks;
         uint32_t out[W / 2];
         uint32_t sb;
         if (!GAIN) {
@@ -243,6 +250,8 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
                 const float y1 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), bf16_hi(gr[j]));
                 my = fmaxf(my, fmaxf(fabsf(y0), fabsf(y1)));
             }
+#pragma unroll
+            for (int o = 1; o < LPB; o <<= 1) my = fmaxf(my, __shfl_xor_sync(0xFFFFFFFFu, my, o));
             sb = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(my) : e8m0_scale(my, P.round);
             const float inv = inv_scale(sb);
 #pragma unroll
@@ -262,14 +271,14 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
 #pragma unroll
                 for (int v = 0; v < W / 16; ++v) st_v8(cp + v * 32, &out[v * 8]);
             }
-            sp0[i * sstep] = (uint8_t)sb;
+            if (LPB == 1 || (lane & (LPB - 1)) == 0) sp0[i * sstep] = (uint8_t)sb;
         }
     }
 }
 
 // phase 2 (MXFP4: E2M1 codes two per byte, E8M0 scales; the paper's rounding rule with 4 = 2^2 as the
 // largest power of two of the element format): S = 2^(ceil(log2 a) - 2)
-template <int B, int NPASS, int WPR>
+template <int B, int NPASS, int WPR, int LPB = 1>
 __device__ __forceinline__ void quantise_store_mxfp4(const uint32_t (&xr)[NPASS][B / 2], const float (&m)[NPASS], float rho,
                                                      const FwdParams& P, int64_t row, int w, int lane)
 {
@@ -277,12 +286,12 @@ __device__ __forceinline__ void quantise_store_mxfp4(const uint32_t (&xr)[NPASS]
     const bool rho_normal = is_normal_f32(rho);
     uint8_t* cp0 = P.codes + row * (P.D / 2) + (int64_t)(w * kWarp + lane) * (B / 2);
     int64_t soff, sstep;
-    scale_addressing<WPR>(P, row, w, lane, soff, sstep);
+    scale_addressing<WPR, LPB>(P, row, w, lane, soff, sstep);
     uint8_t* sp0 = P.scales + soff;
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
         const int k = (i * WPR + w) * kWarp + lane;
-        const bool active = k < P.K;
+        const bool active = k < P.chunks;
         const float a = __fmul_rn(m[i], rho);
         const uint32_t u = __float_as_uint(a), E = u >> 23;
         uint32_t sb;
@@ -314,7 +323,7 @@ __device__ __forceinline__ void quantise_store_mxfp4(const uint32_t (&xr)[NPASS]
             if (B == 16) st_v2(cp, out);
             else if (B == 32) st_v4(cp, out);
             else st_v8(cp, out);
-            sp0[i * sstep] = (uint8_t)sb;
+            if (LPB == 1 || (lane & (LPB - 1)) == 0) sp0[i * sstep] = (uint8_t)sb;
         }
     }
 }
@@ -393,7 +402,7 @@ __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], co
     }
 }
 
-template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER>
+template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER, int LPB = 1>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m3_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
@@ -405,8 +414,8 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m
 
     uint32_t xr[NPASS][B / 2];
     float m[NPASS];
-    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
-    double stat = block_stats<B, NPASS, STAT>(xr, m, P.p);
+    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
+    double stat = block_stats<B, NPASS, STAT, LPB>(xr, m, P.p, lane);
     if (STAT == STAT_RMS) forget_unpacked<NPASS, B / 2>(xr);
     float r = 1.0f, rho = 1.0f;
     if (STAT != STAT_NONE) {
@@ -414,7 +423,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m
         finish_stat<STAT>(stat, P, r, rho);
         if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     }
-    quantise_store_e4m3<B, NPASS, WPR, GAIN, PAPER>(xr, m, rho, P, row, w, lane);
+    quantise_store_e4m3<B, NPASS, WPR, GAIN, PAPER, 0, LPB>(xr, m, rho, P, row, w, lane);
 }
 
 // Residual add fused in front of MXNorm: h = bf16(x + res) is written out as the new residual stream and
@@ -428,7 +437,7 @@ __device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b)
     return d;
 }
 
-template <int B, int NPASS, int WPR>
+template <int B, int NPASS, int WPR, int LPB = 1>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_add_mx_kernel(const FwdParams P)
 {
     constexpr int W = B / 2;
@@ -441,32 +450,32 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_add
 
     uint32_t xr[NPASS][W];
     float m[NPASS];
-    load_row_direct<B, NPASS, true>(xr, P.x + row * P.D, P.K, WPR, w, lane);   // h_out may alias x or residual
+    load_row_direct<B, NPASS, true>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);   // h_out may alias x or residual
     {
         uint32_t rr[NPASS][W];
-        load_row_direct<B, NPASS, true>(rr, P.residual + row * P.D, P.K, WPR, w, lane);
+        load_row_direct<B, NPASS, true>(rr, P.residual + row * P.D, P.chunks, WPR, w, lane);
         uint16_t* hrow = P.h_out + row * P.D;
 #pragma unroll
         for (int i = 0; i < NPASS; ++i) {
 #pragma unroll
             for (int j = 0; j < W; ++j) xr[i][j] = add_bf16x2(xr[i][j], rr[i][j]);
             const int k = (i * WPR + w) * kWarp + lane;
-            if (k < P.K) {
+            if (k < P.chunks) {
 #pragma unroll
                 for (int v = 0; v < W / 8; ++v) st_v8(hrow + (int64_t)k * B + v * 16, &xr[i][v * 8]);
             }
         }
     }
-    double stat = block_stats<B, NPASS, STAT_MX>(xr, m, P.p);
+    double stat = block_stats<B, NPASS, STAT_MX, LPB>(xr, m, P.p, lane);
     stat = group_sum<WPR>(stat, group, w, red);
     float r, rho;
     finish_stat<STAT_MX>(stat, P, r, rho);
     if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
-    quantise_store_e4m3<B, NPASS, WPR, false, true>(xr, m, rho, P, row, w, lane);
+    quantise_store_e4m3<B, NPASS, WPR, false, true, 0, LPB>(xr, m, rho, P, row, w, lane);
 }
 
 // plain MXCast to E5M2 codes (gradient tensors), the paper's rounding rule with 2^15
-template <int B, int NPASS, int WPR>
+template <int B, int NPASS, int WPR, int LPB = 1>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) cast_e5m2_kernel(const FwdParams P)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -476,13 +485,13 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) cast_e5
     if (row >= P.T) return;
     uint32_t xr[NPASS][B / 2];
     float m[NPASS];
-    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
-    (void)block_stats<B, NPASS, STAT_NONE>(xr, m, 2);
-    quantise_store_e4m3<B, NPASS, WPR, false, true, 2>(xr, m, 1.0f, P, row, w, lane);
+    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
+    (void)block_stats<B, NPASS, STAT_NONE, LPB>(xr, m, 2, lane);
+    quantise_store_e4m3<B, NPASS, WPR, false, true, 2, LPB>(xr, m, 1.0f, P, row, w, lane);
 }
 
 // E2M1 codes with E8M0 scales (MXFP4): no gain, the paper's rounding rule
-template <int B, int NPASS, int WPR, int STAT>
+template <int B, int NPASS, int WPR, int STAT, int LPB = 1>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxfp4_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
@@ -494,8 +503,8 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxf
 
     uint32_t xr[NPASS][B / 2];
     float m[NPASS];
-    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
-    double stat = block_stats<B, NPASS, STAT>(xr, m, P.p);
+    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
+    double stat = block_stats<B, NPASS, STAT, LPB>(xr, m, P.p, lane);
     if (STAT == STAT_RMS) forget_unpacked<NPASS, B / 2>(xr);
     float r = 1.0f, rho = 1.0f;
     if (STAT != STAT_NONE) {
@@ -503,7 +512,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxf
         finish_stat<STAT>(stat, P, r, rho);
         if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
     }
-    quantise_store_mxfp4<B, NPASS, WPR>(xr, m, rho, P, row, w, lane);
+    quantise_store_mxfp4<B, NPASS, WPR, LPB>(xr, m, rho, P, row, w, lane);
 }
 
 template <int NPASS, int WPR, int STAT>
@@ -518,7 +527,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
 
     uint32_t xr[NPASS][8];
     float m[NPASS];
-    load_row_direct<16, NPASS>(xr, P.x + row * P.D, P.K, WPR, w, lane);
+    load_row_direct<16, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
     double stat = block_stats<16, NPASS, STAT>(xr, m, P.p);
     if (STAT == STAT_RMS) forget_unpacked<NPASS, 8>(xr);
     stat = group_sum<WPR>(stat, group, w, red);
@@ -531,126 +540,129 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
 // ---- dispatch ---------------------------------------------------------------------------------
 typedef void (*fwd_fn)(const FwdParams);
 
-// The headline kernels (B = 32 or NVFP4, no gain, the paper's rounding rule) exist for every number of
+// In the templates below B is the number of elements a lane holds per pass and LPB the lanes per block
+// (block size of the format = B * LPB: 16 = 16x1, 32 = 32x1, 64 = 32x2).
+// The headline kernels (E4M3 codes or NVFP4, no gain, the paper's rounding rule) exist for every number of
 // warps per row in kFineWpr, so that hidden sizes of the form {3,5,7} * 2^r fill their lanes; the
 // other variants exist for power-of-two warps per row only.
 static const int kFineWpr[] = {1, 2, 3, 4, 5, 6, 7, 8, 16};
 static const int kCoarseWpr[] = {1, 2, 4, 8, 16};
 
-template <int B, int NPASS, int STAT, bool GAIN, bool PAPER, bool FINE>
+template <int B, int LPB, int NPASS, int STAT, bool GAIN, bool PAPER, bool FINE>
 static fwd_fn e4m3_by_wpr(int wpr)
 {
     switch (wpr) {
-        case 1: return fwd_e4m3_kernel<B, NPASS, 1, STAT, GAIN, PAPER>;
-        case 2: return fwd_e4m3_kernel<B, NPASS, 2, STAT, GAIN, PAPER>;
-        case 4: return fwd_e4m3_kernel<B, NPASS, 4, STAT, GAIN, PAPER>;
-        case 8: return fwd_e4m3_kernel<B, NPASS, 8, STAT, GAIN, PAPER>;
-        case 16: return fwd_e4m3_kernel<B, NPASS, 16, STAT, GAIN, PAPER>;
+        case 1: return fwd_e4m3_kernel<B, NPASS, 1, STAT, GAIN, PAPER, LPB>;
+        case 2: return fwd_e4m3_kernel<B, NPASS, 2, STAT, GAIN, PAPER, LPB>;
+        case 4: return fwd_e4m3_kernel<B, NPASS, 4, STAT, GAIN, PAPER, LPB>;
+        case 8: return fwd_e4m3_kernel<B, NPASS, 8, STAT, GAIN, PAPER, LPB>;
+        case 16: return fwd_e4m3_kernel<B, NPASS, 16, STAT, GAIN, PAPER, LPB>;
         default: break;
     }
     if constexpr (FINE) {
         switch (wpr) {
-            case 3: return fwd_e4m3_kernel<B, NPASS, 3, STAT, GAIN, PAPER>;
-            case 5: return fwd_e4m3_kernel<B, NPASS, 5, STAT, GAIN, PAPER>;
-            case 6: return fwd_e4m3_kernel<B, NPASS, 6, STAT, GAIN, PAPER>;
-            case 7: return fwd_e4m3_kernel<B, NPASS, 7, STAT, GAIN, PAPER>;
+            case 3: return fwd_e4m3_kernel<B, NPASS, 3, STAT, GAIN, PAPER, LPB>;
+            case 5: return fwd_e4m3_kernel<B, NPASS, 5, STAT, GAIN, PAPER, LPB>;
+            case 6: return fwd_e4m3_kernel<B, NPASS, 6, STAT, GAIN, PAPER, LPB>;
+            case 7: return fwd_e4m3_kernel<B, NPASS, 7, STAT, GAIN, PAPER, LPB>;
             default: break;
         }
     }
     return nullptr;
 }
 
-// FINE variants exist for every pass count; the others for WPR = 1 with any pass count and for
-// WPR > 1 with the full pass count only.
-template <int B, int STAT, bool GAIN, bool PAPER>
+// Every variant exists for WPR = 1 with any pass count and for WPR > 1 with the full pass count; the FINE
+// ones also for WPR > 1 with one pass and (four-pass kernels) with two.
+template <int B, int LPB, int STAT, bool GAIN, bool PAPER>
 static fwd_fn pick_e4m3(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    constexpr bool FINE = B == 32 && !GAIN && PAPER && STAT != STAT_POSTROUND;
-    if (FINE || wpr > 1) {
-        if (npass == MAXP) return e4m3_by_wpr<B, MAXP, STAT, GAIN, PAPER, FINE>(wpr);
-        if (FINE && npass == 1) return e4m3_by_wpr<B, 1, STAT, GAIN, PAPER, FINE>(wpr);
+    constexpr bool FINE = !GAIN && PAPER && STAT != STAT_POSTROUND;
+    if (wpr > 1) {
+        if (npass == MAXP) return e4m3_by_wpr<B, LPB, MAXP, STAT, GAIN, PAPER, FINE>(wpr);
+        if (FINE && MAXP >= 4 && npass == MAXP / 2) return e4m3_by_wpr<B, LPB, (MAXP >= 4 ? MAXP / 2 : 1), STAT, GAIN, PAPER, FINE>(wpr);
+        if (FINE && npass == 1) return e4m3_by_wpr<B, LPB, 1, STAT, GAIN, PAPER, FINE>(wpr);
         return nullptr;
     }
     switch (npass) {
-        case 1: return fwd_e4m3_kernel<B, 1, 1, STAT, GAIN, PAPER>;
-        case 2: return fwd_e4m3_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, GAIN, PAPER>;
-        case 3: return fwd_e4m3_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, GAIN, PAPER>;
-        default: return fwd_e4m3_kernel<B, MAXP, 1, STAT, GAIN, PAPER>;
+        case 1: return fwd_e4m3_kernel<B, 1, 1, STAT, GAIN, PAPER, LPB>;
+        case 2: return fwd_e4m3_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, GAIN, PAPER, LPB>;
+        case 3: return fwd_e4m3_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, GAIN, PAPER, LPB>;
+        default: return fwd_e4m3_kernel<B, MAXP, 1, STAT, GAIN, PAPER, LPB>;
     }
 }
-template <int B, bool PAPER>
+template <int B, int LPB, bool PAPER>
 static fwd_fn pick_stat(int stat, bool gain, int wpr, int npass)
 {
     switch (stat) {
-        case STAT_NONE: return pick_e4m3<B, STAT_NONE, false, PAPER>(wpr, npass);
-        case STAT_RMS: return gain ? pick_e4m3<B, STAT_RMS, true, PAPER>(wpr, npass) : pick_e4m3<B, STAT_RMS, false, PAPER>(wpr, npass);
-        case STAT_MX: return gain ? pick_e4m3<B, STAT_MX, true, PAPER>(wpr, npass) : pick_e4m3<B, STAT_MX, false, PAPER>(wpr, npass);
-        case STAT_POSTROUND: return (gain || !PAPER) ? nullptr : pick_e4m3<B, STAT_POSTROUND, false, true>(wpr, npass);
+        case STAT_NONE: return pick_e4m3<B, LPB, STAT_NONE, false, PAPER>(wpr, npass);
+        case STAT_RMS: return gain ? pick_e4m3<B, LPB, STAT_RMS, true, PAPER>(wpr, npass) : pick_e4m3<B, LPB, STAT_RMS, false, PAPER>(wpr, npass);
+        case STAT_MX: return gain ? pick_e4m3<B, LPB, STAT_MX, true, PAPER>(wpr, npass) : pick_e4m3<B, LPB, STAT_MX, false, PAPER>(wpr, npass);
+        case STAT_POSTROUND: return (gain || !PAPER) ? nullptr : pick_e4m3<B, LPB, STAT_POSTROUND, false, true>(wpr, npass);
         default: return nullptr;
     }
 }
-template <int B>
+template <int B, int LPB>
 static fwd_fn pick_round(int round, int stat, bool gain, int wpr, int npass)
 {
-    return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, true>(stat, gain, wpr, npass) : pick_stat<B, false>(stat, gain, wpr, npass);
+    return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, LPB, true>(stat, gain, wpr, npass) : pick_stat<B, LPB, false>(stat, gain, wpr, npass);
 }
-template <int B, int STAT>
+template <int B, int LPB, int STAT>
 static fwd_fn pick_mxfp4(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr == 2) return fwd_mxfp4_kernel<B, MAXP, 2, STAT>;
-    if (wpr == 4) return fwd_mxfp4_kernel<B, MAXP, 4, STAT>;
-    if (wpr == 8) return fwd_mxfp4_kernel<B, MAXP, 8, STAT>;
-    if (wpr == 16) return fwd_mxfp4_kernel<B, MAXP, 16, STAT>;
+    if (wpr == 2) return fwd_mxfp4_kernel<B, MAXP, 2, STAT, LPB>;
+    if (wpr == 4) return fwd_mxfp4_kernel<B, MAXP, 4, STAT, LPB>;
+    if (wpr == 8) return fwd_mxfp4_kernel<B, MAXP, 8, STAT, LPB>;
+    if (wpr == 16) return fwd_mxfp4_kernel<B, MAXP, 16, STAT, LPB>;
     if (wpr != 1) return nullptr;
     switch (npass) {
-        case 1: return fwd_mxfp4_kernel<B, 1, 1, STAT>;
-        case 2: return fwd_mxfp4_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT>;
-        case 3: return fwd_mxfp4_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT>;
-        default: return fwd_mxfp4_kernel<B, MAXP, 1, STAT>;
+        case 1: return fwd_mxfp4_kernel<B, 1, 1, STAT, LPB>;
+        case 2: return fwd_mxfp4_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, LPB>;
+        case 3: return fwd_mxfp4_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, LPB>;
+        default: return fwd_mxfp4_kernel<B, MAXP, 1, STAT, LPB>;
     }
 }
-template <int B>
+template <int B, int LPB>
 static fwd_fn pick_add_mx(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr == 2) return fwd_add_mx_kernel<B, MAXP, 2>;
-    if (wpr == 4) return fwd_add_mx_kernel<B, MAXP, 4>;
-    if (wpr == 8) return fwd_add_mx_kernel<B, MAXP, 8>;
-    if (wpr == 16) return fwd_add_mx_kernel<B, MAXP, 16>;
+    if (wpr == 2) return fwd_add_mx_kernel<B, MAXP, 2, LPB>;
+    if (wpr == 4) return fwd_add_mx_kernel<B, MAXP, 4, LPB>;
+    if (wpr == 8) return fwd_add_mx_kernel<B, MAXP, 8, LPB>;
+    if (wpr == 16) return fwd_add_mx_kernel<B, MAXP, 16, LPB>;
     if (wpr != 1) return nullptr;
     switch (npass) {
-        case 1: return fwd_add_mx_kernel<B, 1, 1>;
-        case 2: return fwd_add_mx_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1>;
-        case 3: return fwd_add_mx_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1>;
-        default: return fwd_add_mx_kernel<B, MAXP, 1>;
+        case 1: return fwd_add_mx_kernel<B, 1, 1, LPB>;
+        case 2: return fwd_add_mx_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, LPB>;
+        case 3: return fwd_add_mx_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, LPB>;
+        default: return fwd_add_mx_kernel<B, MAXP, 1, LPB>;
     }
 }
 
-template <int B>
+template <int B, int LPB>
 static fwd_fn pick_e5m2(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr == 2) return cast_e5m2_kernel<B, MAXP, 2>;
-    if (wpr == 4) return cast_e5m2_kernel<B, MAXP, 4>;
-    if (wpr == 8) return cast_e5m2_kernel<B, MAXP, 8>;
-    if (wpr == 16) return cast_e5m2_kernel<B, MAXP, 16>;
+    if (wpr == 2) return cast_e5m2_kernel<B, MAXP, 2, LPB>;
+    if (wpr == 4) return cast_e5m2_kernel<B, MAXP, 4, LPB>;
+    if (wpr == 8) return cast_e5m2_kernel<B, MAXP, 8, LPB>;
+    if (wpr == 16) return cast_e5m2_kernel<B, MAXP, 16, LPB>;
     if (wpr != 1) return nullptr;
     switch (npass) {
-        case 1: return cast_e5m2_kernel<B, 1, 1>;
-        case 2: return cast_e5m2_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1>;
-        case 3: return cast_e5m2_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1>;
-        default: return cast_e5m2_kernel<B, MAXP, 1>;
+        case 1: return cast_e5m2_kernel<B, 1, 1, LPB>;
+        case 2: return cast_e5m2_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, LPB>;
+        case 3: return cast_e5m2_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, LPB>;
+        default: return cast_e5m2_kernel<B, MAXP, 1, LPB>;
     }
 }
 
-template <int B>
+template <int B, int LPB>
 static fwd_fn pick_mxfp4_stat(int stat, int wpr, int npass)
 {
-    if (stat == STAT_MX) return pick_mxfp4<B, STAT_MX>(wpr, npass);
-    if (stat == STAT_RMS) return pick_mxfp4<B, STAT_RMS>(wpr, npass);
-    return pick_mxfp4<B, STAT_NONE>(wpr, npass);
+    if (stat == STAT_MX) return pick_mxfp4<B, LPB, STAT_MX>(wpr, npass);
+    if (stat == STAT_RMS) return pick_mxfp4<B, LPB, STAT_RMS>(wpr, npass);
+    return pick_mxfp4<B, LPB, STAT_NONE>(wpr, npass);
 }
 
 template <int NPASS, int STAT>
@@ -679,10 +691,11 @@ static fwd_fn pick_nvfp4(int wpr, int npass)
     return nullptr;
 }
 
-// Splits the K blocks of a row over WPR warps x NPASS passes (at most MXN_FWD_MAX_ELEMS elements per
-// lane), choosing among the instantiated kernels by the fraction of idle lanes, with a handicap for
-// splits that use fewer passes than the maximum (more warps, hence more synchronisation, per row:
-// measured at D = 7168, where 4 warps x 2 passes at 87.5 % beat 7 warps x 1 pass at 100 %).
+// Splits the K per-lane pieces of a row (B elements each) over WPR warps x NPASS passes (at most MXN_FWD_MAX_ELEMS
+// elements per lane), choosing among the instantiated kernels by the fraction of idle lanes, with a handicap for
+// splits that leave a lane little work when a row spans several warps (more warps, hence more synchronisation,
+// per row).  Measured at 16384 rows: D = 7168, B = 32: 4 warps x 2 passes at 87.5 % beat 7 warps x 1 pass at 100 %;
+// D = 2560, B = 16: 5 warps x 1 pass (16 elements per lane) at 100 % lost to 2 warps x 4 passes at 62.5 %.
 static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
 {
     const int maxp = MXN_FWD_MAX_ELEMS / B;
@@ -693,11 +706,13 @@ static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
     for (int wi = 0; wi < nw; ++wi) {
         const int w = wl[wi];
         for (int p = maxp; p >= 1; --p) {
-            const bool exists = nvfp4 ? (p == maxp || p == maxp / 2 || p == 1)
-                                      : fine ? (p == maxp || p == 1) : (w == 1 || p == maxp);
+            const bool reduced = p == 1 || (maxp >= 4 && p == maxp / 2);
+            const bool exists = p == maxp || (nvfp4 ? reduced : (w == 1 || (fine && reduced)));
             const long lanes = (long)32 * w * p;
             if (!exists || lanes < K) continue;
-            const double cost = (double)(lanes - K) / (double)lanes + ((p < maxp && w > 1) ? 0.15 : 0.0);
+            const int elems = p * B;   // per lane
+            const double handicap = w == 1 || elems >= MXN_FWD_MAX_ELEMS ? 0.0 : elems >= MXN_FWD_MAX_ELEMS / 2 ? 0.15 : 0.45;
+            const double cost = (double)(lanes - K) / (double)lanes + handicap;
             if (best_cost < 0.0 || cost < best_cost - 1e-9) {
                 best_cost = cost;
                 best_w = w;
@@ -715,7 +730,8 @@ bool fwd_shape_supported(int64_t D, int B)
 {
     if (!(B == 16 || B == 32 || B == 64) || D <= 0 || D % B != 0 || D / B > (1 << 20)) return false;
     int wpr, npass;
-    return plan_row((int)(D / B), B, false, false, &wpr, &npass);   // the coarse set is the narrowest
+    const int E = B == 64 ? 32 : B;
+    return plan_row((int)(D / E), E, false, false, &wpr, &npass);   // the coarse set is the narrowest
 }
 
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
@@ -723,10 +739,12 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
     const bool e5m2 = P.elem == ELEM_E5M2;
     const bool add = P.residual != nullptr;
-    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && !add && stat != STAT_POSTROUND && B == 32 && P.gain == nullptr &&
+    const int E = B == 64 ? 32 : B;   // elements per lane and pass; a block of 64 is shared by two lanes
+    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && !add && stat != STAT_POSTROUND && P.gain == nullptr &&
                                 P.round == MXN_ROUND_RCEIL_POW2);
     P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
-    if (!plan_row(P.K, B, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
+    P.chunks = P.K * (B / E);
+    if (!plan_row(P.chunks, E, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
     {
         const int count = stat == STAT_RMS ? P.D : P.K;   // divisor of the row statistic
@@ -734,15 +752,16 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     }
     const int warps = cta_warps(P.wpr);
     P.rows_per_cta = rows_per_cta(P.wpr);
+    const bool has_gain = P.gain != nullptr;
     fwd_fn fn = nullptr;
     if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
-    else if (add) fn = B == 16 ? pick_add_mx<16>(P.wpr, P.npass) : B == 32 ? pick_add_mx<32>(P.wpr, P.npass) : pick_add_mx<64>(P.wpr, P.npass);
-    else if (e5m2) fn = B == 16 ? pick_e5m2<16>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32>(P.wpr, P.npass) : pick_e5m2<64>(P.wpr, P.npass);
-    else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16>(stat, P.wpr, P.npass)
-                       : B == 32 ? pick_mxfp4_stat<32>(stat, P.wpr, P.npass) : pick_mxfp4_stat<64>(stat, P.wpr, P.npass);
-    else if (B == 16) fn = pick_round<16>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
-    else if (B == 32) fn = pick_round<32>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
-    else fn = pick_round<64>(P.round, stat, P.gain != nullptr, P.wpr, P.npass);
+    else if (add) fn = B == 16 ? pick_add_mx<16, 1>(P.wpr, P.npass) : B == 32 ? pick_add_mx<32, 1>(P.wpr, P.npass) : pick_add_mx<32, 2>(P.wpr, P.npass);
+    else if (e5m2) fn = B == 16 ? pick_e5m2<16, 1>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32, 1>(P.wpr, P.npass) : pick_e5m2<32, 2>(P.wpr, P.npass);
+    else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16, 1>(stat, P.wpr, P.npass)
+                       : B == 32 ? pick_mxfp4_stat<32, 1>(stat, P.wpr, P.npass) : pick_mxfp4_stat<32, 2>(stat, P.wpr, P.npass);
+    else if (B == 16) fn = pick_round<16, 1>(P.round, stat, has_gain, P.wpr, P.npass);
+    else if (B == 32) fn = pick_round<32, 1>(P.round, stat, has_gain, P.wpr, P.npass);
+    else fn = pick_round<32, 2>(P.round, stat, has_gain, P.wpr, P.npass);
     if (fn == nullptr) return cudaErrorInvalidValue;
     const int64_t ctas = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
     if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;

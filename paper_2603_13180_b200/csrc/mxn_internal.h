@@ -25,6 +25,7 @@ struct FwdParams {
     int elem;               // ELEM_E4M3 (one byte per element) or ELEM_E2M1 (two elements per byte)
     // filled by the launcher
     int wpr, npass, rows_per_cta, tiles_per_row;
+    int chunks;             // per-lane pieces of a row: K * (lanes per block)
     int pr_table;           // post-round estimator: index of the block size's f^-1 table
     double inv_count;       // 1/K (MXNorm) or 1/D (RMSNorm) when that is a power of two (exact), else 0
 };

@@ -62,7 +62,7 @@ def test_rmsnorm_mxfp8_fwd_matches_oracle(binding, oracle, T, D):
 
 
 @pytest.mark.parametrize("block", [16, 64])
-@pytest.mark.parametrize("T,D", [(3, 64), (19, 1024), (7, 4096), (4, 8192), (3, 16384)])
+@pytest.mark.parametrize("T,D", [(3, 64), (19, 1024), (5, 2048), (9, 2560), (6, 3072), (7, 4096), (4, 8192), (3, 16384)])
 def test_other_block_sizes(binding, oracle, T, D, block):
     x, gain = rows(T, D, seed=T + D + block)
     got = gu.run_fwd(binding, oracle, "mx", x, block=block, eps=1e-5)
@@ -73,6 +73,9 @@ def test_other_block_sizes(binding, oracle, T, D, block):
     gu.assert_exact(got, gu.run_ref(oracle, "cast", x, block=block), f"mx_cast B={block}")
     got = gu.run_fwd(binding, oracle, "rms", x, gain, block=block, eps=1e-5)
     gu.assert_within_rounding_of_rho(got, gu.run_ref(oracle, "rms", x, gain, block=block, eps=1e-5), block, "rms")
+    for layout in (0, 1):
+        got = gu.run_fwd(binding, oracle, "mx", x, gain, block=block, eps=1e-5, layout=layout)
+        gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, block=block, eps=1e-5), f"mxnorm with gain B={block} layout={layout}")
 
 
 @pytest.mark.parametrize("rnd", [1, 2])
