@@ -126,9 +126,39 @@ def time_launches(fn, n_sets: int, steps: int, warmup: int, stream) -> float:
     return start.elapsed_time(end) / steps
 
 
-def time_small_configs(mx, args, stream):
+def time_graph_replay(fn, n_sets: int, steps: int, warmup: int, stream) -> float:
+    """Like time_launches, but the `steps` launches are captured once into a CUDA graph and the replay is
+    timed: kernels of a few microseconds are otherwise limited by the host's launch rate."""
+    for i in range(warmup):
+        fn(i % n_sets)
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=stream):
+        for i in range(steps):
+            fn(i % n_sets)
+    graph.replay()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record(stream)
+    graph.replay()
+    end.record(stream)
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / steps
+
+
+def time_small_configs(mx, args, main_stream):
     """Forward kernels on the small parity configs C1 [2048,768] and C2 [16384,2048] (context: C1 is
-    launch- and L2-bound, 4.8 MB in all)."""
+    launch- and L2-bound, 4.8 MB in all): direct launches ("ms") and the replay of a CUDA graph of the same
+    launches ("ms_graph")."""
+    stream = torch.cuda.Stream()        # a side stream: the default stream cannot be captured
+    stream.wait_stream(main_stream)
+    with torch.cuda.stream(stream):
+        out = _time_small_configs(mx, args, stream)
+    main_stream.wait_stream(stream)
+    return out
+
+
+def _time_small_configs(mx, args, stream):
     out = {}
     L, sh = mx.lib, stream.cuda_stream
     for name in ("C1", "C2"):
@@ -155,7 +185,9 @@ def time_small_configs(mx, args, stream):
         res = {}
         for kname, fn in (("mxnorm_fwd", fwd), ("rmsnorm_mxfp8_fwd", rms), ("mx_cast", cast)):
             ms = time_launches(fn, sets, args.steps, args.warmup, stream)
-            res[kname] = {"ms": ms, "gbs": nbytes / ms / 1e6, "tokens_per_s": T / (ms * 1e-3)}
+            ms_graph = time_graph_replay(fn, sets, args.steps, args.warmup, stream)
+            res[kname] = {"ms": ms, "gbs": nbytes / ms / 1e6, "tokens_per_s": T / (ms * 1e-3),
+                          "ms_graph": ms_graph, "gbs_graph": nbytes / ms_graph / 1e6}
         res["buffer_sets"] = sets
         out[name] = res
         del xs, outs

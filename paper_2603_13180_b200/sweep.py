@@ -4,6 +4,8 @@ folded away; speed-up of `mxnorm_fwd` over the fused conventional path `rmsnorm_
 over the grid.  Both sides are this library's hand-written kernels on the same GPU (the paper compares two
 torch.compile kernels on a GB200).
 
+Each case is timed as the replay of a CUDA graph of back-to-back launches over rotating buffer sets (3x L2).
+
     python -m paper_2603_13180_b200.sweep [--blocks 32] [--elem e4m3|e2m1|nvfp4] [--tokens 4096 16384 65536] [--json out.json]
 """
 from __future__ import annotations
@@ -21,21 +23,42 @@ HIDDEN = sorted({k * 2 ** r for k in (1, 3, 5, 7) for r in range(4, 15) if 2 ** 
 EPS = 1e-5
 
 
-def _time(fn, sets, steps, warmup, stream):
+def _time(fn, sets, steps, warmup, stream, graph=True):
+    """Microseconds per launch over `steps` back-to-back launches that rotate over `sets` buffer sets.
+    With graph=True the launches are captured once into a CUDA graph and the replay is timed, so that
+    kernels of a few microseconds are not limited by the host's launch rate."""
     for i in range(warmup):
         fn(i % sets)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    a.record(stream)
-    for i in range(steps):
-        fn(i % sets)
-    b.record(stream)
+    if graph:
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(steps):
+                fn(i % sets)
+        g.replay()                     # untimed: uploads the graph
+        torch.cuda.synchronize()
+        a.record(stream)
+        g.replay()
+        b.record(stream)
+    else:
+        torch.cuda.synchronize()
+        a.record(stream)
+        for i in range(steps):
+            fn(i % sets)
+        b.record(stream)
     torch.cuda.synchronize()
     return a.elapsed_time(b) / steps * 1e3   # microseconds
 
 
-def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4m3"):
-    stream = torch.cuda.current_stream()
+def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4m3", graph=True):
+    stream = torch.cuda.Stream()       # a side stream: the default stream cannot be captured
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        return _run(stream, tokens, hidden, blocks, steps, warmup, l2_bytes, elem, graph)
+
+
+def _run(stream, tokens, hidden, blocks, steps, warmup, l2_bytes, elem, graph):
     sh = stream.cuda_stream
     L = mx.lib
     rows = []
@@ -84,8 +107,8 @@ def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4
                                              0, mx.SCALES_SWIZZLE_128x4, sh)
                     assert st == 0, mx.status_string(st)
 
-                t_mx = min(_time(mxn, sets, steps, warmup, stream) for _ in range(2))
-                t_rms = min(_time(rms, sets, steps, warmup, stream) for _ in range(2))
+                t_mx = min(_time(mxn, sets, steps, warmup, stream, graph) for _ in range(2))
+                t_rms = min(_time(rms, sets, steps, warmup, stream, graph) for _ in range(2))
                 rows.append({"elem": elem, "block": B, "tokens": T, "hidden": D, "mxnorm_us": t_mx, "rmsnorm_us": t_rms,
                              "speedup": t_rms / t_mx, "mxnorm_gbs": per_set / t_mx / 1e3, "rmsnorm_gbs": per_set / t_rms / 1e3})
                 del xs, outs
@@ -115,9 +138,10 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--elem", default="e4m3", choices=["e4m3", "e2m1", "nvfp4"],
                     help="element format: e4m3/e2m1 with E8M0 scales, or nvfp4 (E2M1 codes, E4M3 scales, block 16)")
+    ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a CUDA-graph replay")
     ap.add_argument("--json", default="")
     args = ap.parse_args()
-    rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps, elem=args.elem)
+    rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps, elem=args.elem, graph=not args.no_graph)
     summary = summarise(rows)
     for r in rows:
         print(f"{r['elem']} B={r['block']:2d} T={r['tokens']:6d} D={r['hidden']:6d}  mxnorm {r['mxnorm_us']:9.2f} us {r['mxnorm_gbs']:6.0f} GB/s   "
