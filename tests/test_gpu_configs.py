@@ -45,6 +45,16 @@ def test_mxfp8_configs_full_size(binding, oracle, name):
         gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, eps=EPS), f"{name} mxnorm_fwd with gain")
 
 
+@pytest.mark.parametrize("block", [16, 64])
+def test_other_block_sizes_at_the_benchmark_shape(binding, oracle, block):
+    """[16384, 4096] with blocks of 16 and 64 (two lanes share a block of 64), E4M3 and E2M1 codes, tiled scales."""
+    x = wl.bits(wl.make_inputs(wl.CONFIGS["C3"])["x"])
+    got = gu.run_fwd(binding, oracle, "mx", x, block=block, eps=EPS, layout=1)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", x, block=block, eps=EPS), f"mxnorm_fwd B={block}")
+    got = gu.run_fwd(binding, oracle, "mx4", x, block=block, eps=EPS, layout=1)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx4", x, block=block, eps=EPS), f"mxnorm_mxfp4_fwd B={block}")
+
+
 def test_nvfp4_config_full_size(binding, oracle):
     w = wl.CONFIGS["C4"]
     x = wl.bits(wl.make_inputs(w)["x"])
