@@ -13,6 +13,18 @@
 
 namespace mxn {
 
+// Token tiles are spread over grid dimensions y and z (y alone is limited to 65535 tiles); ZSPILL selects the kernels
+// that read blockIdx.z (the common case, z = 1, keeps the two-dimensional code: measured 1.5 % faster at [16384,4096])
+constexpr unsigned kMaxGridY = 65535;
+template <bool ZSPILL>
+__device__ __forceinline__ unsigned token_tile_index() { return ZSPILL ? blockIdx.z * kMaxGridY + blockIdx.y : blockIdx.y; }
+static dim3 token_tile_grid(int64_t col_tiles, int64_t token_tiles)
+{
+    const int64_t z = (token_tiles + kMaxGridY - 1) / kMaxGridY;
+    return dim3((unsigned)col_tiles, (unsigned)(z > 1 ? kMaxGridY : token_tiles), (unsigned)z);
+}
+
+
 __device__ __forceinline__ uint2 ld_v2(const void* p)
 {
     uint2 r;
@@ -26,12 +38,12 @@ __device__ __forceinline__ uint2 ld_v2(const void* p)
 constexpr int kTrCpl = MXN_TR_CPL;
 constexpr int kTrTileCols = 32 * kTrCpl;
 
-template <bool PAPER, int ELEM>
+template <bool PAPER, int ELEM, bool ZSPILL>
 __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedParams P)
 {
     constexpr int CPL = kTrCpl, WORDS = CPL / 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t t0 = ((int64_t)blockIdx.y * 4 + warp) * 32;
+    const int64_t t0 = ((int64_t)token_tile_index<ZSPILL>() * 4 + warp) * 32;
     const int c0 = blockIdx.x * kTrTileCols + lane * CPL;
     pdl_prologue();
     if (t0 >= P.T) return;
@@ -145,7 +157,7 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-template <bool PAPER, int ELEM>
+template <bool PAPER, int ELEM, bool ZSPILL>
 __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_kernel(const TransposedParams P)
 {
     extern __shared__ __align__(128) uint8_t tile_raw[];
@@ -153,7 +165,7 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t tile0 = (uint32_t)__cvta_generic_to_shared(tile_raw);
     const int ctile = blockIdx.x * kTsCols;                  // first column of the CTA's tile
-    const int64_t tbase = (int64_t)blockIdx.y * kTsTpc * 32;   // first token of the CTA
+    const int64_t tbase = (int64_t)token_tile_index<ZSPILL>() * kTsTpc * 32;   // first token of the CTA
     pdl_prologue();
 
     auto issue = [&](int tt) {
@@ -250,13 +262,14 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
 {
     P.KT = (int)(P.T / 32);
     P.tiles_per_row = (P.KT + 3) / 4;
+    // grid: x = column tiles, (y, z) = token tiles (more than kMaxGridY of them spill into z; CTAs past the end leave at once)
     const int64_t gx = (P.D + kTrTileCols - 1) / kTrTileCols, gy = (P.T + 127) / 128;
-    if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
+    if (gx > 0x7FFFFFFF || (gy + kMaxGridY - 1) / kMaxGridY > 65535) return cudaErrorInvalidValue;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)gx, (unsigned)gy);
+    cfg.gridDim = token_tile_grid(gx, gy);
     cfg.blockDim = dim3(128);
     cfg.stream = stream;
     cfg.attrs = attr;
@@ -264,22 +277,26 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
 #ifndef MXN_TR_NO_SMEM
     if (P.D % 8 == 0) {   // 16-byte row chunks: the shared-memory staged kernel
         const int64_t sx = (P.D + kTsCols - 1) / kTsCols, sy = (P.T / 32 + kTsTpc - 1) / kTsTpc;
-        if (sy <= 65535) {
-            auto kfn = P.elem == ELEM_E5M2 ? cast_transposed_smem_kernel<true, 2>
-                       : P.round == MXN_ROUND_RCEIL_POW2 ? cast_transposed_smem_kernel<true, 0> : cast_transposed_smem_kernel<false, 0>;
+        if ((sy + kMaxGridY - 1) / kMaxGridY <= 65535) {
+            const bool zs = sy > kMaxGridY;
+            auto kfn = P.elem == ELEM_E5M2 ? (zs ? cast_transposed_smem_kernel<true, 2, true> : cast_transposed_smem_kernel<true, 2, false>)
+                       : P.round == MXN_ROUND_RCEIL_POW2 ? (zs ? cast_transposed_smem_kernel<true, 0, true> : cast_transposed_smem_kernel<true, 0, false>)
+                                                         : (zs ? cast_transposed_smem_kernel<false, 0, true> : cast_transposed_smem_kernel<false, 0, false>);
             const int smem = kTsStages * kTsStageBytes;
             const cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
             if (e != cudaSuccess) return e;
-            cfg.gridDim = dim3((unsigned)sx, (unsigned)sy);
+            cfg.gridDim = token_tile_grid(sx, sy);
             cfg.blockDim = dim3(kTsThreads);
             cfg.dynamicSmemBytes = smem;
             return cudaLaunchKernelEx(&cfg, kfn, P);
         }
     }
 #endif
-    if (P.elem == ELEM_E5M2) return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<true, 2>, P);
-    if (P.round == MXN_ROUND_RCEIL_POW2) return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<true, 0>, P);
-    return cudaLaunchKernelEx(&cfg, cast_transposed_kernel<false, 0>, P);
+    const bool zs = gy > kMaxGridY;
+    auto kfn = P.elem == ELEM_E5M2 ? (zs ? cast_transposed_kernel<true, 2, true> : cast_transposed_kernel<true, 2, false>)
+               : P.round == MXN_ROUND_RCEIL_POW2 ? (zs ? cast_transposed_kernel<true, 0, true> : cast_transposed_kernel<true, 0, false>)
+                                                 : (zs ? cast_transposed_kernel<false, 0, true> : cast_transposed_kernel<false, 0, false>);
+    return cudaLaunchKernelEx(&cfg, kfn, P);
 }
 
 }  // namespace mxn

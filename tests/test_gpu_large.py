@@ -64,3 +64,24 @@ def test_forward_and_backward_beyond_2_31_elements(binding, oracle):
         wct, wst = oracle.mx_cast_transposed_ref(blk, rms=rms[t0:t0 + 32].cpu().numpy(), eps=1e-5)
         assert np.array_equal(ct[cols, t0:t0 + 32].cpu().numpy(), wct[cols])
         assert np.array_equal(st.view(D, T2 // 32)[cols, t0 // 32].cpu().numpy(), wst[cols, 0])
+
+
+def test_token_counts_beyond_65535_tiles(binding, oracle):
+    """Very long, narrow tensors: more than 65535 token tiles in the column-wise cast and more than 2^21 rows in the
+    row-wise kernels (grids are one-dimensional, so only the total number of CTAs is bounded)."""
+    T, D = 65537 * 32, 64                        # 2,097,184 tokens
+    x = _big_input(T, D, seed=9)
+    codes, scales, rms = binding.alloc_outputs(T, D, 32, binding.SCALES_ROWMAJOR)
+    binding.mxnorm_fwd(x, None, codes, scales, rms, eps=1e-5)
+    ct = torch.empty((D, T), dtype=torch.uint8, device="cuda")
+    st = torch.empty((D, T // 32), dtype=torch.uint8, device="cuda")
+    binding.mx_cast_transposed(x, rms, ct, st, eps=1e-5)
+    torch.cuda.synchronize()
+    xb = wl.bits(x.cpu())
+    wc, ws, wr = oracle.mxnorm_ref(xb, eps=1e-5)
+    assert np.array_equal(codes.cpu().numpy(), wc)
+    assert np.array_equal(scales.cpu().numpy().reshape(T, D // 32), ws)
+    assert np.array_equal(rms.cpu().numpy(), wr)
+    wct, wst = oracle.mx_cast_transposed_ref(xb, rms=wr, eps=1e-5)
+    assert np.array_equal(ct.cpu().numpy(), wct)
+    assert np.array_equal(st.cpu().numpy(), wst)
