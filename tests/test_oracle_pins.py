@@ -537,6 +537,12 @@ def test_postround_estimator(oracle):
     xs = bf16_bits(bf16_vals(x[:32]) * np.float32(2.0 ** -7))
     c1, s1, r1 = oracle.mxnorm_postround_ref(xs)
     assert np.array_equal(c0, c1) and np.array_equal(s0, s1) and np.array_equal(r1, r0 * np.float32(2.0 ** -7))
+    # eps enters as rho~ = 1/(r~ + eps): with eps = r~ the denominator doubles exactly, so every scale exponent
+    # drops by one, the codes stay and the reported r~ does not include eps
+    for t in (0, 5):
+        c0, s0, r0 = oracle.mxnorm_postround_ref(x[t:t + 1])
+        c1, s1, r1 = oracle.mxnorm_postround_ref(x[t:t + 1], eps=float(r0[0]))
+        assert np.array_equal(r1, r0) and np.array_equal(c1, c0) and np.array_equal(s1.astype(int), s0.astype(int) - 1)
     z = np.zeros((1, 64), np.uint16)
     c, s_, r = oracle.mxnorm_postround_ref(z, eps=1e-5)
     assert np.all(c == 0) and np.all(s_ == 0) and r[0] == 0
