@@ -10,6 +10,7 @@
 // 128 contiguous bytes per CTA.  Every input byte is read once, every output byte written once.
 #include "mxn_device.cuh"
 #include "mxn_internal.h"
+#include "mxn_col.cuh"
 
 namespace mxn {
 
@@ -209,50 +210,10 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
 #pragma unroll
         for (int r = 0; r < 32; ++r) asm volatile("ld.shared.b32 %0, [%1];" : "=r"(xr[r]) : "r"(wordaddr + (uint32_t)r * kTsRowBytes));
 
-        float m0 = 0.f, m1 = 0.f;
-#pragma unroll
-        for (int r = 0; r < 32; r += 4) {
-            const float4 r4 = *reinterpret_cast<const float4*>(rho + r);   // broadcast read
-            const float rv[4] = {r4.x, r4.y, r4.z, r4.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 y = mul2(bf16x2_to_f32x2(xr[r + i]), make_float2(rv[i], rv[i]));
-                m0 = fmaxf(m0, fabsf(y.x));
-                m1 = fmaxf(m1, fabsf(y.y));
-            }
-        }
-        const uint32_t sb0 = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(m0) : e8m0_scale(m0, P.round);
-        const uint32_t sb1 = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(m1) : e8m0_scale(m1, P.round);
-        const float2 inv = make_float2(inv_scale(sb0), inv_scale(sb1));
-        uint32_t out0[8], out1[8];
-#pragma unroll
-        for (int r = 0; r < 32; r += 4) {
-            float2 q[4];
-            const float4 r4 = *reinterpret_cast<const float4*>(rho + r);
-            const float rv[4] = {r4.x, r4.y, r4.z, r4.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) q[i] = mul2(mul2(bf16x2_to_f32x2(xr[r + i]), make_float2(rv[i], rv[i])), inv);
-            out0[r / 4] = cvt_fp8x4<ELEM>(q[0].x, q[1].x, q[2].x, q[3].x);
-            out1[r / 4] = cvt_fp8x4<ELEM>(q[0].y, q[1].y, q[2].y, q[3].y);
-        }
+        uint32_t out0[8], out1[8], sb0, sb1;
+        quantise_column_pair<PAPER, ELEM>(xr, rho, P.round, out0, out1, sb0, sb1);
         const int c = ctile + (warp * 32 + lane) * 2;
-        if (c < P.D) {
-            const int k = (int)(t0 >> 5);
-            st_v8(P.codes + (int64_t)c * P.T + t0, out0);
-            st_v8(P.codes + (int64_t)(c + 1) * P.T + t0, out1);
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int64_t row = c + j;
-                int64_t off;
-                if (P.layout == MXN_SCALES_ROWMAJOR) {
-                    off = row * P.KT + k;
-                } else {
-                    const int rr = (int)(row & 127);
-                    off = ((row >> 7) * P.tiles_per_row + (k >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (k & 3);
-                }
-                P.scales[off] = (uint8_t)(j == 0 ? sb0 : sb1);
-            }
-        }
+        if (c < P.D) store_column_pair(P.codes, P.scales, P.T, P.KT, P.tiles_per_row, P.layout, c, t0, out0, out1, sb0, sb1);
         __syncthreads();   // the stage may be refilled by the next issue()
     }
     cp_async_wait<0>();
