@@ -477,6 +477,14 @@ def main():
 
         msb = time_launches(bwd, nb, max(10, args.steps // 2), args.warmup, stream)
         others["mxnorm_bwd"] = {"ms": msb, "gbs": algorithmic_bytes("bwd", T, D) / msb / 1e6}
+
+        def bwd_dx_only(i):   # the method's own configuration: no gain (folded into the next weight), hence no gain gradient
+            st = L.mxnorm_bwd(xb[i].data_ptr(), gb[i].data_ptr(), None, rmsb.data_ptr(), T, D, dxb[i].data_ptr(), 0, None, None, 0, sh)
+            if st != 0:
+                raise RuntimeError(mx.status_string(st))
+
+        msbx = time_launches(bwd_dx_only, nb, max(10, args.steps // 2), args.warmup, stream)
+        others["mxnorm_bwd_dx_only"] = {"ms": msbx, "gbs": (3 * T * D * 2 + 4 * T) / msbx / 1e6}
         del xb, gb, dxb
         for v in others.values():
             v["frac_of_peak"] = v["gbs"] / peak
