@@ -60,3 +60,49 @@ def test_block_scaled_gemm_consumes_tiled_scales(oracle, T, D, N):
                                out_dtype=torch.bfloat16)
         bad_err = (bad.double() - ref).abs().max().item() / ref.abs().max().item()
         assert bad_err > 10 * err
+
+
+@pytest.mark.parametrize("T,D,N", [(256, 512, 128), (512, 1024, 256), (384, 768, 96)])
+def test_weight_gradient_gemm_consumes_the_column_wise_casts(oracle, T, D, N):
+    """The weight gradient of Section 3.7, grad W = MXCast(grad H^T) MXCast(rho~ X), contracts over the TOKENS: both
+    operands are the [*, T] outputs of mx_cast_transposed with their tiled scales, handed to the block-scaled GEMM as
+    they are.  Pins the transposed outputs' layout against the consumer."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_13180_b200 import binding as mx
+    if not hasattr(torch, "_scaled_mm") or not hasattr(torch, "float8_e8m0fnu"):
+        pytest.skip("this torch has no block-scaled matmul")
+    tiled = mx.SCALES_SWIZZLE_128x4
+    inp = wl.make_inputs(wl.Workload("t", T, D, seed=T + D + N, outlier_frac=0.002))
+    x = inp["x"].cuda()
+    g = torch.Generator(device="cpu").manual_seed(N)
+    grad_h = (1e-2 * torch.randn(T, N, generator=g)).to(torch.bfloat16).cuda()
+
+    # forward: r~ per token; then the two column-wise casts
+    cx, sx, rms = mx.alloc_outputs(T, D, 32, tiled)
+    mx.mxnorm_fwd(x, None, cx, sx, rms, eps=1e-5, layout=tiled)
+    KT = T // 32
+    xt = torch.empty((D, T), dtype=torch.uint8, device="cuda")
+    xts = torch.empty(mx.scale_bytes(D, KT, tiled), dtype=torch.uint8, device="cuda")
+    mx.mx_cast_transposed(x, rms, xt, xts, eps=1e-5, layout=tiled)
+    gt = torch.empty((N, T), dtype=torch.uint8, device="cuda")
+    gts = torch.empty(mx.scale_bytes(N, KT, tiled), dtype=torch.uint8, device="cuda")
+    mx.mx_cast_transposed(grad_h, None, gt, gts, layout=tiled)
+    try:
+        out = torch._scaled_mm(gt.view(torch.float8_e4m3fn), xt.view(torch.float8_e4m3fn).t(),
+                               scale_a=gts.view(torch.float8_e8m0fnu), scale_b=xts.view(torch.float8_e8m0fnu),
+                               out_dtype=torch.bfloat16)
+    except (RuntimeError, NotImplementedError) as e:
+        pytest.skip(f"torch._scaled_mm rejected MXFP8 block scales: {str(e)[:120]}")
+    torch.cuda.synchronize()
+
+    gts_rm = torch.from_numpy(gts.cpu().numpy()[oracle.swizzle_index_map(N, KT)]).cuda()
+    xts_rm = torch.from_numpy(xts.cpu().numpy()[oracle.swizzle_index_map(D, KT)]).cuda()
+    a, b = _dequant(gt, gts_rm, N, T), _dequant(xt, xts_rm, D, T)          # [N, T] and [D, T], blocks along T
+    ref = a @ b.t()
+    err = (out.double() - ref).abs().max().item() / ref.abs().max().item()
+    assert err < 1e-2, err
+    # and the quantised product is the weight gradient of the unquantised operands to MXFP8 accuracy
+    rho = 1.0 / (rms.double() + 1e-5)
+    exact = grad_h.double().t() @ (x.double() * rho[:, None])
+    assert (ref - exact).abs().max().item() < 0.08 * exact.abs().max().item()
