@@ -106,3 +106,47 @@ def test_weight_gradient_gemm_consumes_the_column_wise_casts(oracle, T, D, N):
     rho = 1.0 / (rms.double() + 1e-5)
     exact = grad_h.double().t() @ (x.double() * rho[:, None])
     assert (ref - exact).abs().max().item() < 0.08 * exact.abs().max().item()
+
+
+_E2M1 = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+
+
+def _dequant_nvfp4(codes_packed, scales_rowmajor_e4m3, T, D):
+    """[T, D/2] bytes (low nibble = even element) and E4M3 scale bytes [T, D/16] -> [T, D] binary64"""
+    lut = torch.tensor(_E2M1 + [-v for v in _E2M1], dtype=torch.float64, device=codes_packed.device)
+    lo, hi = (codes_packed & 0xF).long(), (codes_packed >> 4).long()
+    vals = torch.stack([lut[lo], lut[hi]], dim=-1).view(T, D // 16, 16)
+    sc = scales_rowmajor_e4m3.view(torch.float8_e4m3fn).double().view(T, D // 16, 1)
+    return (vals * sc).view(T, D)
+
+
+@pytest.mark.parametrize("T,D,N", [(256, 512, 128), (384, 4096, 256)])
+def test_nvfp4_gemm_consumes_packed_codes_and_e4m3_scales(oracle, T, D, N):
+    """NVFP4 (which the paper does not define beyond block 16 / E2M1): the packed nibbles and the tiled E4M3 block scales
+    that mxnorm_nvfp4_fwd emits are what the block-scaled FP4 GEMM of the vendor library expects - nibble order, scale
+    format and scale layout pinned against that consumer."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2603_13180_b200 import binding as mx
+    if not hasattr(torch, "_scaled_mm") or not hasattr(torch, "float4_e2m1fn_x2"):
+        pytest.skip("this torch has no FP4 block-scaled matmul")
+    tiled = mx.SCALES_SWIZZLE_128x4
+    x = wl.make_inputs(wl.Workload("t", T, D, seed=T + D, outlier_frac=0.002))["x"].cuda()
+    w = wl.make_inputs(wl.Workload("w", N, D, seed=N + D))["x"].cuda()
+    cx, sx, _ = mx.alloc_outputs(T, D, 16, tiled, nvfp4=True)
+    cw, sw, _ = mx.alloc_outputs(N, D, 16, tiled, nvfp4=True)
+    mx.mxnorm_nvfp4_fwd(x, cx, sx, None, eps=1e-5, layout=tiled)
+    mx.mxnorm_nvfp4_fwd(w, cw, sw, None, eps=1e-5, layout=tiled)        # any NVFP4 tensor serves as the second operand
+    try:
+        out = torch._scaled_mm(cx.view(torch.float4_e2m1fn_x2), cw.view(torch.float4_e2m1fn_x2).t(),
+                               scale_a=sx.view(torch.float8_e4m3fn), scale_b=sw.view(torch.float8_e4m3fn),
+                               out_dtype=torch.bfloat16)
+    except (RuntimeError, NotImplementedError, TypeError) as e:
+        pytest.skip(f"torch._scaled_mm rejected NVFP4 operands: {str(e)[:160]}")
+    torch.cuda.synchronize()
+    K = D // 16
+    sx_rm = torch.from_numpy(sx.cpu().numpy()[oracle.swizzle_index_map(T, K)]).cuda()
+    sw_rm = torch.from_numpy(sw.cpu().numpy()[oracle.swizzle_index_map(N, K)]).cuda()
+    ref = _dequant_nvfp4(cx, sx_rm, T, D) @ _dequant_nvfp4(cw, sw_rm, N, D).t()
+    err = (out.double() - ref).abs().max().item() / ref.abs().max().item()
+    assert err < 1e-2, err
