@@ -12,9 +12,9 @@ from paper_2603_13180_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-def _dequant(codes, scales_rowmajor, T, D):
+def _dequant(codes, scales_rowmajor, T, D, elem=torch.float8_e4m3fn):
     K = D // 32
-    vals = codes.view(torch.float8_e4m3fn).float().view(T, K, 32)
+    vals = codes.view(elem).float().view(T, K, 32)
     return (vals * torch.exp2(scales_rowmajor.view(T, K, 1).float() - 127.0)).view(T, D).double()
 
 
@@ -62,8 +62,9 @@ def test_block_scaled_gemm_consumes_tiled_scales(oracle, T, D, N):
         assert bad_err > 10 * err
 
 
+@pytest.mark.parametrize("grad_e5m2", [False, True])
 @pytest.mark.parametrize("T,D,N", [(256, 512, 128), (512, 1024, 256), (384, 768, 96)])
-def test_weight_gradient_gemm_consumes_the_column_wise_casts(oracle, T, D, N):
+def test_weight_gradient_gemm_consumes_the_column_wise_casts(oracle, T, D, N, grad_e5m2):
     """The weight gradient of Section 3.7, grad W = MXCast(grad H^T) MXCast(rho~ X), contracts over the TOKENS: both
     operands are the [*, T] outputs of mx_cast_transposed with their tiled scales, handed to the block-scaled GEMM as
     they are.  Pins the transposed outputs' layout against the consumer."""
@@ -87,18 +88,22 @@ def test_weight_gradient_gemm_consumes_the_column_wise_casts(oracle, T, D, N):
     mx.mx_cast_transposed(x, rms, xt, xts, eps=1e-5, layout=tiled)
     gt = torch.empty((N, T), dtype=torch.uint8, device="cuda")
     gts = torch.empty(mx.scale_bytes(N, KT, tiled), dtype=torch.uint8, device="cuda")
-    mx.mx_cast_transposed(grad_h, None, gt, gts, layout=tiled)
+    gdt = torch.float8_e5m2 if grad_e5m2 else torch.float8_e4m3fn       # E5M2: the option the paper names for gradients
+    if grad_e5m2:
+        mx.mx_cast_transposed_e5m2(grad_h, gt, gts, layout=tiled)
+    else:
+        mx.mx_cast_transposed(grad_h, None, gt, gts, layout=tiled)
     try:
-        out = torch._scaled_mm(gt.view(torch.float8_e4m3fn), xt.view(torch.float8_e4m3fn).t(),
+        out = torch._scaled_mm(gt.view(gdt), xt.view(torch.float8_e4m3fn).t(),
                                scale_a=gts.view(torch.float8_e8m0fnu), scale_b=xts.view(torch.float8_e8m0fnu),
                                out_dtype=torch.bfloat16)
     except (RuntimeError, NotImplementedError) as e:
-        pytest.skip(f"torch._scaled_mm rejected MXFP8 block scales: {str(e)[:120]}")
+        pytest.skip(f"torch._scaled_mm rejected these MXFP8 operands: {str(e)[:120]}")
     torch.cuda.synchronize()
 
     gts_rm = torch.from_numpy(gts.cpu().numpy()[oracle.swizzle_index_map(N, KT)]).cuda()
     xts_rm = torch.from_numpy(xts.cpu().numpy()[oracle.swizzle_index_map(D, KT)]).cuda()
-    a, b = _dequant(gt, gts_rm, N, T), _dequant(xt, xts_rm, D, T)          # [N, T] and [D, T], blocks along T
+    a, b = _dequant(gt, gts_rm, N, T, gdt), _dequant(xt, xts_rm, D, T)     # [N, T] and [D, T], blocks along T
     ref = a @ b.t()
     err = (out.double() - ref).abs().max().item() / ref.abs().max().item()
     assert err < 1e-2, err
