@@ -12,7 +12,7 @@
  *    allocates, frees or synchronises; work is enqueued on `cuda_stream` (a
  *    cudaStream_t passed as void*, NULL = the legacy default stream) of the
  *    device that is current when the call is made.
- *  - X is bf16 [T, D], row-major, contiguous, base address 16-byte aligned.
+ *  - X is bf16 [T, D], row-major, contiguous, base address 32-byte aligned (read with 32-byte loads).
  *    T >= 0 rows (tokens), D hidden size, `block` = B, K = D / B blocks per row.
  *    Supported: B in {16, 32, 64} (NVFP4: B = 16 fixed), D % B == 0,
  *    D <= 32768 (backward: D % 8 == 0, D <= 16384).  T == 0 returns MXN_OK without a launch.
