@@ -52,6 +52,8 @@ def _load():
         lib.mxnorm_bwd_ref.argtypes = [vp, vp, vp, vp, i64, i64, vp, vp]
         lib.rmsnorm_nvfp4_ref.argtypes = [vp, i64, i64, f32, f32, vp, vp, vp]
         lib.rmsnorm_nvfp4_ref.restype = i32
+        lib.nvfp4_cast_ref.argtypes = [vp, i64, i64, f32, vp, vp]
+        lib.nvfp4_cast_ref.restype = i32
         lib.mxnorm_postround_ref.argtypes = [vp, i64, i64, i32, f32, i32, vp, vp, vp]
         lib.mxnorm_postround_ref.restype = i32
         lib.mxnorm_add_ref.argtypes = [vp, vp, i64, i64, i32, i32, f32, f32, i32, vp, vp, vp, vp]
@@ -175,6 +177,16 @@ def rmsnorm_nvfp4_ref(x, eps=0.0, global_scale=1.0):
     _check(_load().rmsnorm_nvfp4_ref(_p(x), T, D, eps, global_scale, _p(codes), _p(scales), _p(rms)),
            "rmsnorm_nvfp4_ref")
     return codes, scales, rms
+
+
+def nvfp4_cast_ref(x, global_scale=1.0):
+    """Plain NVFP4 cast (no normalisation): returns (packed codes [T, D/2] u8, E4M3 scales [T, D/16] u8)."""
+    x = _bf16(x, 2)
+    T, D = x.shape
+    codes = np.zeros((T, D // 2), np.uint8)
+    scales = np.zeros((T, D // 16 if D % 16 == 0 else 0), np.uint8)
+    _check(_load().nvfp4_cast_ref(_p(x), T, D, global_scale, _p(codes), _p(scales)), "nvfp4_cast_ref")
+    return codes, scales
 
 
 def mxnorm_add_ref(x, res, p=2, coef=0.0, eps=0.0, block=32, mode=ROUND_RCEIL_POW2):

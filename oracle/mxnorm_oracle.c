@@ -432,6 +432,31 @@ int mxnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, int p, float 
     return 0;
 }
 
+/* The plain NVFP4 cast (no normalisation: rho = 1), e.g. of a weight matrix: the tail above applied to x itself
+ * [reading, as above; a per-tensor global_scale is the caller's]. */
+int nvfp4_cast_ref(const uint16_t *x_bf16, int64_t T, int64_t D, float global_scale,
+                   uint8_t *codes_packed, uint8_t *scales_e4m3)
+{
+    const int B = 16;
+    if (!shape_ok(T, D, B)) return 1;
+    int64_t K = D / B;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *xr = x_bf16 + t * D;
+        float m[K];
+        for (int64_t k = 0; k < K; ++k) {
+            float mk = 0.0f;
+            for (int b = 0; b < B; ++b) {
+                float a = fabsf(bf16_to_f32(xr[k * B + b]));
+                if (a > mk) mk = a;
+            }
+            m[k] = mk;
+        }
+        nvfp4_quantise_row(xr, m, D, 1.0f, global_scale, codes_packed + t * (D / 2), scales_e4m3 + t * K);
+    }
+    return 0;
+}
+
 /* The conventional counterpart in the same format: Algorithm 1's rho (true RMS) followed by the NVFP4 cast of
  * x * rho [reading, as above].  Block absmaxes of fl32(x*rho) equal fl32(m_k * rho) because rounding is monotone. */
 int rmsnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, float eps, float global_scale,

@@ -356,6 +356,33 @@ def test_nvfp4_scales_and_codes_by_definition_given_rho(oracle):
         assert np.all(np.abs(deq - ynorm) <= 0.25 * np.repeat(a, 16, axis=1) + 1e-6)
 
 
+def test_plain_nvfp4_cast_by_definition(oracle):
+    """The cast without a normaliser (weights): block scale = nearest E4M3 value to absmax/6*g, codes = nearest E2M1 value
+    to x*g/scale, and it is what the normalising variants produce when their rho is 1."""
+    x = wl.bits(wl.make_inputs(wl.Workload("t", 12, 256, seed=8, outlier_frac=0.004))["x"])
+    xv = bf16_vals(x)
+    for gs in (1.0, 0.5, 8.0):
+        codes, scales = oracle.nvfp4_cast_ref(x, global_scale=gs)
+        a = np.abs(xv).reshape(12, -1, 16).max(-1)
+        t = ((a / np.float32(6.0)).astype(np.float32) * np.float32(gs)).astype(np.float32)
+        sc, _ = nearest_code(t.astype(np.float64), E4M3_POS)
+        assert np.array_equal(scales, sc)
+        d = E4M3_POS[sc].astype(np.float32)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            inv = np.where(d == 0, np.float32(0), (np.float32(gs) / d).astype(np.float32))
+        q = (xv * np.repeat(inv, 16, axis=1)).astype(np.float32)
+        code, neg = nearest_code(q.astype(np.float64), E2M1_POS)
+        nib = code | (neg.astype(np.uint8) << 3)
+        assert np.array_equal(codes, nib[:, 0::2] | (nib[:, 1::2] << 4))
+    # a constant row of ones: absmax/6 = 0.16667 -> nearest E4M3 value 0.171875 = 0x23; 1/0.171875 = 5.818 -> 6 -> 0x7
+    ones = np.full((1, 32), ONE, np.uint16)
+    codes, scales = oracle.nvfp4_cast_ref(ones)
+    assert np.all(scales == 0x23) and np.all(codes == 0x77)
+    # the normalising variant with a coefficient that makes r~ = 1 exactly (constant row of ones: G = 1) gives the same bytes
+    c2, s2, r2 = oracle.mxnorm_nvfp4_ref(ones, coef=1.0)
+    assert r2[0] == 1.0 and np.array_equal(c2, codes) and np.array_equal(s2, scales)
+
+
 def test_mxfp4_element_format_by_definition(oracle):
     """E2M1 values with E8M0 scales (the listing's cast with dtype = E2M1): the largest power of two of the
     format is 4, so S is the smallest power of two with absmax/S <= 4; codes are the nearest E2M1 values,
