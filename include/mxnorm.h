@@ -176,6 +176,13 @@ mxn_status rmsnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, float eps
                              void* codes_u8_packed, void* scales_e4m3, float* rms_out_or_null,
                              mxn_scale_layout layout, void* cuda_stream);
 
+/* The NVFP4 cast without a normaliser (rho = 1), e.g. for the weight operand W*gamma of MXNormLinear in the NVFP4
+ * configuration (Section 3.7; the paper does not define NVFP4 beyond block 16 / E2M1, see mxnorm_nvfp4_fwd):
+ * block scale = E4M3(absmax / 6 * global_scale), codes = E2M1(x * global_scale / scale).
+ * Same buffers and conventions as mxnorm_nvfp4_fwd. */
+mxn_status mx_cast_nvfp4(const void* x_bf16, int64_t T, int64_t D, float global_scale,
+                      void* codes_u8_packed, void* scales_e4m3, mxn_scale_layout layout, void* cuda_stream);
+
 /* MXFP4 counterparts of the three forward entry points: E2M1 element values (two per byte, element 2i in
  * the low nibble: codes_u8_packed [T, D/2], 32-byte aligned) with E8M0 block scales, B in {16, 32, 64} -
  * the paper's cast with the element type set to E2M1 (appendix "Implementation of MXNormLinear";

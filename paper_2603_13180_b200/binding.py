@@ -24,7 +24,7 @@ EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd
            "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
            "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
-           "mxnorm_add_fwd")
+           "mxnorm_add_fwd", "mx_cast_nvfp4")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -60,6 +60,7 @@ lib.mxnorm_postround_fwd.argtypes = [_vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp,
 lib.mx_cast_e5m2.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _vp]
 lib.mx_cast_transposed_e5m2.argtypes = [_vp, _i64, _i64, _vp, _vp, _i32, _vp]
 lib.rmsnorm_nvfp4_fwd.argtypes = [_vp, _i64, _i64, _f32, _f32, _vp, _vp, _vp, _i32, _vp]
+lib.mx_cast_nvfp4.argtypes = [_vp, _i64, _i64, _f32, _vp, _vp, _i32, _vp]
 lib.mx_cast_transposed.argtypes = [_vp, _vp, _i64, _i64, _f32, _vp, _vp, _i32, _i32, _vp]
 lib.mxnorm_bwd_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i32, _vp, _vp]
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.argtypes = []
@@ -68,7 +69,7 @@ for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", 
               "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
            "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
-           "mxnorm_add_fwd"):
+           "mxnorm_add_fwd", "mx_cast_nvfp4"):
     getattr(lib, _name).restype = _i32
 
 
@@ -242,6 +243,14 @@ def rmsnorm_nvfp4_fwd(x, codes_packed, scales_e4m3, rms_out=None, eps=0.0, globa
     T, D = x.shape
     _check(lib.rmsnorm_nvfp4_fwd(_ptr(x), T, D, eps, global_scale, _ptr(codes_packed), _ptr(scales_e4m3), _ptr(rms_out),
                                  layout, _stream(stream)), "rmsnorm_nvfp4_fwd")
+
+
+def mx_cast_nvfp4(x, codes_packed, scales_e4m3, global_scale=1.0, layout=SCALES_ROWMAJOR, stream=None):
+    """NVFP4 cast without a normaliser (e.g. of a weight): E2M1 codes two per byte, E4M3 scales per 16 elements."""
+    _dev(x, torch.bfloat16, "x")
+    T, D = x.shape
+    _check(lib.mx_cast_nvfp4(_ptr(x), T, D, global_scale, _ptr(codes_packed), _ptr(scales_e4m3), layout, _stream(stream)),
+           "mx_cast_nvfp4")
 
 
 def mx_cast_e5m2(x, codes, scales, block=32, layout=SCALES_ROWMAJOR, stream=None):

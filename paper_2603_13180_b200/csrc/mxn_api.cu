@@ -153,6 +153,13 @@ mxn_status mxnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int p, flo
                    scales_e4m3, rms_est_out_or_null, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
 }
 
+mxn_status mx_cast_nvfp4(const void* x_bf16, int64_t T, int64_t D, float global_scale, void* codes_u8_packed,
+                      void* scales_e4m3, mxn_scale_layout layout, void* cuda_stream)
+{
+    return run_fwd(mxn::STAT_NONE, true, x_bf16, nullptr, T, D, 16, 2, 1.0f, 0.0f, global_scale, codes_u8_packed,
+                   scales_e4m3, nullptr, MXN_ROUND_RCEIL_POW2, layout, cuda_stream);
+}
+
 mxn_status rmsnorm_nvfp4_fwd(const void* x_bf16, int64_t T, int64_t D, float eps, float global_scale,
                              void* codes_u8_packed, void* scales_e4m3, float* rms_out_or_null,
                              mxn_scale_layout layout, void* cuda_stream)

@@ -176,10 +176,12 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
     load_row_direct<16, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
     double stat = block_stats<16, NPASS, STAT>(xr, m, P.p);
     if (STAT == STAT_RMS) forget_unpacked<NPASS, 8>(xr);
-    stat = group_sum<WPR>(stat, group, w, red);
-    float r, rho;
-    finish_stat<STAT>(stat, P, r, rho);
-    if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    float r = 1.0f, rho = 1.0f;
+    if (STAT != STAT_NONE) {
+        stat = group_sum<WPR>(stat, group, w, red);
+        finish_stat<STAT>(stat, P, r, rho);
+        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    }
     quantise_store_nvfp4<NPASS, WPR>(xr, m, rho, P, row, w, lane);
 }
 
@@ -400,7 +402,7 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     P.rows_per_cta = rows_per_cta(P.wpr);
     const bool has_gain = P.gain != nullptr;
     fwd_fn fn = nullptr;
-    if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
+    if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
     else if (add) fn = B == 16 ? pick_add_mx<16, 1>(P.wpr, P.npass) : B == 32 ? pick_add_mx<32, 1>(P.wpr, P.npass) : pick_add_mx<32, 2>(P.wpr, P.npass);
     else if (e5m2) fn = B == 16 ? pick_e5m2<16, 1>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32, 1>(P.wpr, P.npass) : pick_e5m2<32, 2>(P.wpr, P.npass);
     else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16, 1>(stat, P.wpr, P.npass)

@@ -36,7 +36,7 @@ def run_fwd(binding, oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coe
     T, D = x_bits.shape
     x = wl.from_bits(x_bits).cuda()
     gain = None if gain_bits is None else wl.from_bits(gain_bits).cuda()
-    nvfp4 = kind in ("nvfp4", "rms_nvfp4")
+    nvfp4 = kind in ("nvfp4", "rms_nvfp4", "cast_nvfp4")
     fp4 = nvfp4 or kind in ("cast4", "rms4", "mx4")     # E2M1 codes: two elements per byte
     B = 16 if nvfp4 else block
     K = D // B
@@ -62,6 +62,9 @@ def run_fwd(binding, oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coe
         binding.mxnorm_postround_fwd(x, codes, scales, rms, eps=eps, block=B, layout=layout)
     elif kind == "rms_nvfp4":
         binding.rmsnorm_nvfp4_fwd(x, codes, scales, rms, eps=eps, global_scale=global_scale, layout=layout)
+    elif kind == "cast_nvfp4":
+        binding.mx_cast_nvfp4(x, codes, scales, global_scale=global_scale, layout=layout)
+        rms = None
     elif kind == "cast4":
         binding.mx_cast_fp4(x, codes, scales, block=B, layout=layout)
         rms = None
@@ -99,6 +102,9 @@ def run_ref(oracle, kind, x_bits, gain_bits=None, *, block=32, p=2, coef=0.0, ep
         return oracle.mxnorm_postround_ref(x_bits, eps=eps, block=block)
     if kind == "rms_nvfp4":
         return oracle.rmsnorm_nvfp4_ref(x_bits, eps=eps, global_scale=global_scale)
+    if kind == "cast_nvfp4":
+        c, s = oracle.nvfp4_cast_ref(x_bits, global_scale=global_scale)
+        return c, s, None
     if kind == "cast4":
         c, s = oracle.mx_cast_ref(x_bits, block=block, elem=oracle.ELEM_E2M1)
         return c, s, None

@@ -141,7 +141,7 @@ def test_nvfp4_gemm_consumes_packed_codes_and_e4m3_scales(oracle, T, D, N):
     cx, sx, _ = mx.alloc_outputs(T, D, 16, tiled, nvfp4=True)
     cw, sw, _ = mx.alloc_outputs(N, D, 16, tiled, nvfp4=True)
     mx.mxnorm_nvfp4_fwd(x, cx, sx, None, eps=1e-5, layout=tiled)
-    mx.mxnorm_nvfp4_fwd(w, cw, sw, None, eps=1e-5, layout=tiled)        # any NVFP4 tensor serves as the second operand
+    mx.mx_cast_nvfp4(w, cw, sw, layout=tiled)                               # the weight operand: cast without a normaliser
     try:
         out = torch._scaled_mm(cx.view(torch.float4_e2m1fn_x2), cw.view(torch.float4_e2m1fn_x2).t(),
                                scale_a=sx.view(torch.float8_e4m3fn), scale_b=sw.view(torch.float8_e4m3fn),

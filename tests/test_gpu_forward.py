@@ -162,6 +162,10 @@ def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
         gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x, p=p, eps=eps, global_scale=gs), f"nvfp4 {T}x{D} p={p}")
     got = gu.run_fwd(binding, oracle, "nvfp4", x, layout=1)
     gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x), "nvfp4 tiled scales")
+    # the cast without a normaliser (weights)
+    for gs, layout in ((1.0, 0), (0.25, 1)):
+        got = gu.run_fwd(binding, oracle, "cast_nvfp4", x, global_scale=gs, layout=layout)
+        gu.assert_exact(got, gu.run_ref(oracle, "cast_nvfp4", x, global_scale=gs), f"mx_cast_nvfp4 {T}x{D} g={gs}")
 
 
 def test_power_of_two_shift_on_gpu(binding, oracle):
