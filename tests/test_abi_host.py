@@ -86,3 +86,17 @@ def test_binding_module_has_no_fallback():
     src = open(os.path.join(ROOT, "paper_2603_13180_b200", "binding.py")).read()
     assert "oracle" not in src.replace("CPU oracle", "")
     assert "raise ImportError" in src
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own, with no CUDA or C++ headers."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "mxnorm.h"\n'
+                   "int main(void) { return mxn_scale_bytes(0, 0, MXN_SCALES_ROWMAJOR) == 0 && MXN_OK == 0 ? 0 : 1; }\n")
+    r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only",
+                        "-I", os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
