@@ -100,3 +100,27 @@ def test_header_is_plain_c(tmp_path):
     r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only",
                         "-I", os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
     assert r.returncode == 0, r.stderr
+
+
+def test_library_links_and_runs_from_c(binding, tmp_path):
+    """A C program linked against libmxnorm.so calls the host-only entry points (no GPU needed)."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    libdir = os.path.join(ROOT, "paper_2603_13180_b200")
+    src = tmp_path / "link_test.c"
+    src.write_text('#include <stdio.h>\n#include <string.h>\n#include "mxnorm.h"\n'
+                   "int main(void) {\n"
+                   "    if (mxn_scale_bytes(16384, 128, MXN_SCALES_SWIZZLE_128x4) != 16384u * 128u) return 1;\n"
+                   "    if (mxn_scale_bytes(130, 5, MXN_SCALES_SWIZZLE_128x4) != 2u * 2u * 512u) return 2;\n"
+                   "    if (strlen(mxn_status_string(MXN_ERR_ALIGN)) == 0) return 3;\n"
+                   "    if (mx_cast(0, -1, 4096, 32, 0, 0, MXN_ROUND_RCEIL_POW2, MXN_SCALES_ROWMAJOR, 0) != MXN_ERR_SHAPE) return 4;\n"
+                   "    if (mxnorm_fwd(0, 0, 0, 4096, 32, 2, 0.0f, 0.0f, 0, 0, 0, MXN_ROUND_RCEIL_POW2, MXN_SCALES_ROWMAJOR, 0) != MXN_OK) return 5;\n"
+                   '    puts("ok");\n    return 0;\n}\n')
+    exe = tmp_path / "link_test"
+    r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src),
+                        "-L", libdir, "-lmxnorm", "-Wl,-rpath," + libdir, "-o", str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0 and r.stdout.strip() == "ok", (r.returncode, r.stdout, r.stderr)
