@@ -96,6 +96,10 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
     const float invD = __fdiv_rn(1.0f, (float)P.D);
     const int64_t stride = gridDim.x;
 
+    if (tid < 2 * stages) {   // the first ring fill into L2 before the wait for the previous kernel (see prefetch_l2_bulk)
+        const int64_t row = (int64_t)blockIdx.x + (tid >> 1) * stride;
+        if (row < P.T) prefetch_l2_bulk(((tid & 1) ? P.g : P.x) + row * P.D, row_bytes);
+    }
     pdl_prologue();
     if (tid == 0) {
         abort_flag = 0;

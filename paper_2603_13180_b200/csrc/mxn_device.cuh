@@ -199,6 +199,15 @@ __device__ __forceinline__ bool is_normal_f32(float f)
 // while this one is still running.  Memory is only touched after the wait, so results are the same as
 // with fully serialised launches; what overlaps is the launch latency and block scheduling of one
 // kernel with the tail of the previous one.
+// Hint: bring `bytes` (a multiple of 16, 16-byte aligned address) into L2.  A prefetch consumes no value, so it may be
+// issued BEFORE griddepcontrol.wait: L2 is the point of coherence, a line prefetched early and then written by the
+// previous kernel is simply updated in place, and the loads that follow the wait see the new data.  What it buys: the
+// CTAs of this kernel that become resident while the previous kernel drains fill the idle DRAM with their first rows.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(p), "r"(bytes) : "memory");
+}
+
 __device__ __forceinline__ void pdl_prologue()
 {
     asm volatile("griddepcontrol.wait;" ::: "memory");

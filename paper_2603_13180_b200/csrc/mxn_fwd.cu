@@ -48,6 +48,13 @@ __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], co
     }
 }
 
+// One lane per row asks for the whole row in L2 before the kernel waits for its predecessor (see prefetch_l2_bulk):
+// rows are multiples of 32 bytes and 32-byte aligned.
+__device__ __forceinline__ void prefetch_row(const uint16_t* base, int64_t row, const FwdParams& P, int w, int lane)
+{
+    if (w == 0 && lane == 0 && row < P.T) prefetch_l2_bulk(base + row * P.D, (uint32_t)P.D * 2u);
+}
+
 template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER, int LPB = 1>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m3_kernel(const FwdParams P)
 {
@@ -55,6 +62,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_e4m
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    prefetch_row(P.x, row, P, w, lane);
     pdl_prologue();
     if (row >= P.T) return;   // whole row group leaves together
 
@@ -91,6 +99,8 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_add
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    prefetch_row(P.x, row, P, w, lane);
+    prefetch_row(P.residual, row, P, w, lane);
     pdl_prologue();
     if (row >= P.T) return;
 
@@ -127,6 +137,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) cast_e5
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    prefetch_row(P.x, row, P, w, lane);
     pdl_prologue();
     if (row >= P.T) return;
     uint32_t xr[NPASS][B / 2];
@@ -144,6 +155,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_mxf
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    prefetch_row(P.x, row, P, w, lane);
     pdl_prologue();
     if (row >= P.T) return;
 
@@ -168,6 +180,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
     const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    prefetch_row(P.x, row, P, w, lane);
     pdl_prologue();
     if (row >= P.T) return;
 

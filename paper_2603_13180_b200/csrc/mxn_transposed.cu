@@ -167,6 +167,11 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
     const uint32_t tile0 = (uint32_t)__cvta_generic_to_shared(tile_raw);
     const int ctile = blockIdx.x * kTsCols;                  // first column of the CTA's tile
     const int64_t tbase = (int64_t)token_tile_index<ZSPILL>() * kTsTpc * 32;   // first token of the CTA
+    {   // the first tile into L2 before the wait for the previous kernel (a hint: see prefetch_l2_bulk): one 128-byte line per thread
+        const int row = tid / (kTsRowBytes / 128), part = tid % (kTsRowBytes / 128);
+        if (row < 32 && tbase + row < P.T && ctile + part * 64 < P.D)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(P.x + (tbase + row) * P.D + ctile + part * 64) : "memory");
+    }
     pdl_prologue();
 
     auto issue = [&](int tt) {

@@ -89,3 +89,33 @@ def test_captured_step_replays_bit_exactly(binding, oracle, layout):
     assert np.array_equal(cap["codes_t"].cpu().numpy(), tc)
     if layout == 0:
         assert np.array_equal(cap["scales_t"].cpu().numpy().reshape(D, T // 32), ts)
+
+
+def test_consumer_kernel_right_behind_its_producer(binding, oracle):
+    """Kernels ask for their input rows in L2 before they wait for the previous kernel of the stream.  When that previous
+    kernel is the PRODUCER of those rows the early request may only ever be a hint: here mxnorm_add_fwd writes h and
+    mxnorm_fwd reads h right behind it, at full size and with fresh data every iteration, and the consumer's bytes must be
+    those of the producer's own fused MXNorm of h (and the oracle's on sampled rows)."""
+    T, D = 16384, 4096
+    g = torch.Generator(device="cuda").manual_seed(5)
+    h = torch.empty((T, D), dtype=torch.bfloat16, device="cuda")
+    ca, sa, ra = binding.alloc_outputs(T, D, 32, 1)
+    cb, sb, rb = binding.alloc_outputs(T, D, 32, 1)
+    ct = torch.empty((D, T), dtype=torch.uint8, device="cuda")
+    st = torch.empty(binding.scale_bytes(D, T // 32, 1), dtype=torch.uint8, device="cuda")
+    ct2, st2 = torch.empty_like(ct), torch.empty_like(st)
+    for it in range(12):
+        x = (torch.randn(T, D, generator=g, device="cuda") * (1.0 + it)).to(torch.bfloat16)
+        res = torch.randn(T, D, generator=g, device="cuda").to(torch.bfloat16)
+        torch.cuda.synchronize()
+        binding.mxnorm_add_fwd(x, res, h, ca, sa, ra, eps=1e-5, layout=1)      # producer of h (and of its MXNorm)
+        binding.mxnorm_fwd(h, None, cb, sb, rb, eps=1e-5, layout=1)            # consumer, launched right behind
+        binding.mx_cast_transposed(h, rb, ct, st, eps=1e-5, layout=1)          # second consumer (of h and of rb)
+        torch.cuda.synchronize()
+        assert torch.equal(ca, cb) and torch.equal(sa, sb) and torch.equal(ra.view(torch.int32), rb.view(torch.int32)), it
+        binding.mx_cast_transposed(h, ra, ct2, st2, eps=1e-5, layout=1)        # the same cast with nothing in flight
+        torch.cuda.synchronize()
+        assert torch.equal(ct, ct2) and torch.equal(st, st2), it
+    rows = torch.tensor([0, 1, 4097, T - 1], device="cuda")
+    want_c, _, want_r = oracle.mxnorm_ref(wl.bits(h[rows].cpu()), eps=1e-5)
+    assert np.array_equal(cb[rows].cpu().numpy(), want_c) and np.array_equal(rb[rows].cpu().numpy(), want_r)
