@@ -27,9 +27,11 @@
  *    The buffer must hold mxn_scale_bytes(T, K, layout) bytes; padding bytes are
  *    written as 0.
  *  - Launch semantics: kernels are launched with programmatic stream serialisation.  Each kernel
- *    waits, before its first memory access, until the preceding kernel of the stream has completed and
- *    its writes are visible, so ordering and results are those of ordinary stream order; only the
- *    launch latency of one kernel overlaps the tail of the previous one.  A kernel that FOLLOWS a
+ *    waits, before it reads or writes any value, until the preceding kernel of the stream has completed
+ *    and its writes are visible, so ordering and results are those of ordinary stream order; what
+ *    overlaps the tail of the previous kernel is the launch latency and L2 prefetch hints for the first
+ *    input rows (a prefetch consumes no value; L2 is the point of coherence, so a line requested early
+ *    and then written by the previous kernel is read with its new contents).  A kernel that FOLLOWS a
  *    libmxnorm kernel and is itself launched with the programmatic attribute must do the same wait
  *    (griddepcontrol.wait / cudaGridDependencySynchronize) before reading libmxnorm's outputs;
  *    ordinary launches need nothing.
