@@ -48,11 +48,14 @@ __device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], co
     }
 }
 
+constexpr unsigned kFirstWaveCtas = 148 * 8;   // SMs x the most CTAs of 128 threads an SM holds at 64 registers
+
 // One lane per row asks for the whole row in L2 before the kernel waits for its predecessor (see prefetch_l2_bulk):
 // rows are multiples of 32 bytes and 32-byte aligned.
 __device__ __forceinline__ void prefetch_row(const uint16_t* base, int64_t row, const FwdParams& P, int w, int lane)
 {
-    if (w == 0 && lane == 0 && row < P.T) prefetch_l2_bulk(base + row * P.D, (uint32_t)P.D * 2u);
+    // only CTAs of the first wave can be resident before the previous kernel has ended; for the rest the hint is redundant
+    if (w == 0 && lane == 0 && row < P.T && blockIdx.x < kFirstWaveCtas) prefetch_l2_bulk(base + row * P.D, (uint32_t)P.D * 2u);
 }
 
 template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER, int LPB = 1>

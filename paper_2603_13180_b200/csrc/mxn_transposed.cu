@@ -169,7 +169,8 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
     const int64_t tbase = (int64_t)token_tile_index<ZSPILL>() * kTsTpc * 32;   // first token of the CTA
     {   // the first tile into L2 before the wait for the previous kernel (a hint: see prefetch_l2_bulk): one 128-byte line per thread
         const int row = tid / (kTsRowBytes / 128), part = tid % (kTsRowBytes / 128);
-        if (row < 32 && tbase + row < P.T && ctile + part * 64 < P.D)
+        const bool first_wave = (uint64_t)token_tile_index<ZSPILL>() * gridDim.x < 148u * 16u;   // later CTAs start after the wait is over
+        if (first_wave && row < 32 && tbase + row < P.T && ctile + part * 64 < P.D)
             asm volatile("prefetch.global.L2 [%0];" :: "l"(P.x + (tbase + row) * P.D + ctile + part * 64) : "memory");
     }
     pdl_prologue();
