@@ -367,8 +367,9 @@ def main():
                                "outlier channels, MXFP8 E4M3 codes + E8M0 scales (B=32) in the 128x4 tiled GEMM layout, p=2",
                    "l2": f"inputs/outputs rotate over {SETS} buffer sets ({SETS * nbytes / 1e6:.0f} MB > 126 MB L2)",
                    "launch": "back-to-back launches in one stream, as the library issues them: programmatic stream "
-                             "serialisation (each kernel waits for the previous one before its first memory access; launch "
-                             "latency overlaps the previous kernel's tail); event_between_launches_ms_per_step records an event after every launch",
+                             "serialisation (each kernel waits for the previous one before it reads or writes any value; launch "
+                             "latency and L2 prefetch hints for the first-wave rows overlap the previous kernel's tail); "
+                             "event_between_launches_ms_per_step records an event after every launch",
                    "parallelism": f"rows sharded, no collective (x{world})"},
         "event_between_launches_ms_per_step": ms_serial,
         "tokens_per_s": T * world / (ms * 1e-3),
