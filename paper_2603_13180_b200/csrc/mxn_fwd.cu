@@ -15,7 +15,10 @@
 //     D squares (RMSNorm), reduced in binary64 by shuffles (and through shared memory when a row
 //     spans several warps);
 //   * short-lived CTAs (one per 1-4 rows), launched with programmatic stream serialisation: measured
-//     faster on B200 than resident CTAs, with or without TMA staging.
+//     faster on B200 than resident CTAs, with or without TMA staging;
+//   * the CTAs of the first wave ask for their rows in L2 (a bulk prefetch hint) before they wait for the
+//     previous kernel of the stream, so that the DRAM idling during that kernel's tail already fetches
+//     this kernel's first rows; no value is read before the wait.
 #include <cmath>
 #include <mutex>
 
