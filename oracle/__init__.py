@@ -62,6 +62,8 @@ def _load():
         lib.mxn_ref_postround_f.restype = ctypes.c_double
         lib.mxn_ref_postround_f_inverse.argtypes = [ctypes.c_double, i32]
         lib.mxn_ref_postround_f_inverse.restype = ctypes.c_double
+        lib.mxn_ref_postround_estimate.argtypes = [vp, i64, i32, vp]
+        lib.mxn_ref_postround_estimate.restype = None
         lib.mx_cast_transposed_ref.argtypes = [vp, vp, i64, i64, i32, f32, i32, i32, vp, vp]
         lib.mx_cast_transposed_ref.restype = i32
         for f in (lib.mx_cast_ref, lib.rmsnorm_mxfp8_ref, lib.mxnorm_ref, lib.mxnorm_nvfp4_ref,
@@ -83,8 +85,6 @@ def _load():
         lib.mxn_ref_e5m2_encode.restype = ctypes.c_uint8
         lib.mxn_ref_e8m0_scale.argtypes = [f32, i32, i32]
         lib.mxn_ref_e8m0_scale.restype = ctypes.c_uint8
-        lib.mxn_ref_f64_to_bf16.argtypes = [ctypes.c_double]
-        lib.mxn_ref_f64_to_bf16.restype = ctypes.c_uint16
         lib.mxn_ref_num_threads.restype = i32
         _lib = lib
     return _lib
@@ -224,6 +224,15 @@ def postround_f_inverse(x: float, block: int) -> float:
     return float(_load().mxn_ref_postround_f_inverse(x, block))
 
 
+def postround_estimate(xbar, block: int) -> np.ndarray:
+    """r~ = f^-1(xbar) through the 64-interval table for an array of arguments (binary64, before the rounding to
+    binary32)."""
+    xb = np.ascontiguousarray(np.atleast_1d(xbar), dtype=np.float64)
+    out = np.zeros_like(xb)
+    _load().mxn_ref_postround_estimate(_p(xb), xb.size, block, _p(out))
+    return out
+
+
 def mxnorm_bwd_ref(x, g, gain, rms, want_dx=True, want_dgain=True):
     """Straight-through backward in fp64: returns (dX [T, D] f64 | None, dgain [D] f64 | None)."""
     x = _bf16(x, 2)
@@ -287,7 +296,3 @@ def e5m2_encode(q: float) -> int:
 
 def e8m0_scale(a: float, mode=ROUND_RCEIL_POW2, elem=ELEM_E4M3) -> int:
     return int(_load().mxn_ref_e8m0_scale(a, mode, elem))
-
-
-def f64_to_bf16(v: float) -> int:
-    return int(_load().mxn_ref_f64_to_bf16(v))

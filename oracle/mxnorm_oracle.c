@@ -17,16 +17,19 @@
  * Readings taken where the paper is silent or inconsistent are marked
  * [reading]; the project's design document lists them all.
  *
- * Pin status (see tests/test_oracle_*.py):
- *   mx_cast_ref, rmsnorm_mxfp8_ref, mxnorm_ref, mxnorm_bwd_ref, mx_cast_transposed_ref : pinned
- *     (printed constants and bounds, closed forms, invariants, brute force,
- *      library special cases, finite differences).
- *   mxnorm_nvfp4_ref : PARITY UNPINNED by the paper - the paper gives only
- *     "B = 16, E2M1"; the scale rule is a stated reading, pinned by brute
- *     force and invariants only.
- *   mxn_ref_swizzle_offset : PARITY UNPINNED on the CPU (layout is not in the
- *     paper); pinned on the GPU by feeding a block-scaled GEMM.
+ * Pin status (see tests/test_oracle_pins.py): every function and branch below is pinned by something other
+ * than itself - the paper's printed constants and bounds, closed forms, invariants, brute-force definitional
+ * searches, library special cases (torch casts, scipy's erf and root finder), finite differences.
+ *   mx_cast_ref, rmsnorm_mxfp8_ref, mxnorm_ref (with and without gain), mxnorm_bwd_ref, mx_cast_transposed_ref,
+ *   mxnorm_add_ref, mxnorm_postround_ref (series, inverse, table and interpolation against an independent
+ *   scipy/numpy restatement) : pinned.
+ *   mxnorm_nvfp4_ref, rmsnorm_nvfp4_ref, nvfp4_cast_ref : the paper gives only "B = 16, E2M1"; the scale rule is
+ *     a stated reading, so these are PARITY UNPINNED BY THE PAPER and pinned by the definitional search,
+ *     closed forms and invariants of that reading only.
+ *   mxn_ref_swizzle_offset : the tiled scale layout is not in the paper; structural pin on the CPU, pinned
+ *     against a block-scaled GEMM on the GPU.
  */
+#include <float.h>
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -51,27 +54,16 @@ static float bf16_to_f32(uint16_t h)
     return f;
 }
 
-/* round-to-nearest-even of a binary64 to bf16 bits (used only for dX output) */
-static uint16_t f64_to_bf16(double v)
+/* rho = 1/den in binary32, for the normalisation factors rho~ = 1/(r~ + eps) and rho = 1/r.
+ * den == 0 gives 0 (a zero row stays zero) [reading].  A denominator so small that the
+ * reciprocal would overflow binary32 (den < 2^-128: rows of subnormal magnitude) gives the
+ * largest finite binary32 instead of infinity [reading: the reciprocal saturates, as the
+ * element casts do], so that no 0 * inf = NaN can arise from finite input. */
+static float recip_sat(float den)
 {
-    /* rounds the double directly (going through fp32 first would round twice) */
-    if (isnan(v)) return 0x7FC0;
-    uint16_t sign = signbit(v) ? 0x8000 : 0;
-    double a = fabs(v);
-    if (a == 0.0) return sign;
-    if (isinf(a)) return sign | 0x7F80;
-    int ex;
-    (void)frexp(a, &ex);          /* a = f * 2^ex, f in [0.5,1) -> floor(log2 a) = ex-1 */
-    int e = ex - 1;
-    if (e < -126) e = -126;       /* subnormal quantum */
-    double quantum = ldexp(1.0, e - 7);
-    double n = rint(a / quantum); /* exact division by a power of two; RN-even */
-    double r = n * quantum;
-    if (r >= ldexp(1.0, 128)) return sign | 0x7F80;
-    float rf = (float)r;          /* exactly representable */
-    uint32_t u;
-    memcpy(&u, &rf, 4);
-    return sign | (uint16_t)(u >> 16);
+    if (den == 0.0f) return 0.0f;
+    float rho = 1.0f / den;
+    return rho > FLT_MAX ? FLT_MAX : rho;
 }
 
 /* cast(q; E4M3): OCP "fn" flavour - bias 7, 3 mantissa bits, subnormals down to
@@ -299,7 +291,7 @@ int rmsnorm_mxfp8_ref(const uint16_t *x_bf16, const uint16_t *gain_bf16, int64_t
         }
         double ms = ss / (double)D;
         float r = (float)sqrt(ms + (double)eps);
-        float rho = r == 0.0f ? 0.0f : 1.0f / r;
+        float rho = recip_sat(r);
         float y[D];
         for (int64_t d = 0; d < D; ++d) {
             float v = bf16_to_f32(xr[d]) * rho;
@@ -328,7 +320,8 @@ float mxn_ref_coef(int B, int p)
 /* steps 1-3 of Algorithm 2 for one row: block absmaxes m_k (exact), the
  * generalised p-mean G = (1/K sum m_k^p)^(1/p) in fp64 (Eq. G_K^(p)), the RMS
  * estimate r~ = fl32(coef * G) [reading: coef = RMS/G < 1 multiplies G], and
- * rho~ = fl32(1 / fl32(r~ + eps)), 0 when the denominator is 0 [reading]. */
+ * rho~ = fl32(1 / fl32(r~ + eps)), 0 when the denominator is 0 and saturating at the largest
+ * finite binary32 (recip_sat) [reading]. */
 static void mxnorm_row_stat(const uint16_t *xr, int64_t D, int B, int p, float coef, float eps,
                             float *m /* [K] */, float *r_est, float *rho)
 {
@@ -347,7 +340,7 @@ static void mxnorm_row_stat(const uint16_t *xr, int64_t D, int B, int p, float c
     float rt = (float)((double)coef * G);
     float den = rt + eps;
     *r_est = rt;
-    *rho = den == 0.0f ? 0.0f : 1.0f / den;
+    *rho = recip_sat(den);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -388,7 +381,9 @@ int mxnorm_ref(const uint16_t *x_bf16, const uint16_t *gain_bf16, int64_t T, int
 /*     steps 1-3 with B = 16; a_k = fl32(m_k*rho~);                            */
 /*     t_k = fl32(fl32(a_k / 6) * global_scale); block scale = cast(t_k; E4M3) */
 /*     (6 = largest E2M1 value); d_k = the decoded scale;                      */
-/*     inv_k = fl32(fl32(rho~ * global_scale) / d_k) (0 when d_k = 0);         */
+/*     inv_k = fl32(fl32(rho~ * global_scale) / d_k) (0 when d_k = 0), saturating */
+/*     at the largest finite binary32 [reading, as for rho~ itself: a quotient  */
+/*     that overflowed to infinity would turn zero elements into NaN];         */
 /*     V_kb = cast(fl32(x_kb * inv_k); E2M1), two codes per byte.              */
 /* ------------------------------------------------------------------------- */
 /* shared NVFP4 tail: given the row's block absmaxes m_k of |x| and rho, emit E4M3 block scales and E2M1 codes */
@@ -405,6 +400,7 @@ static void nvfp4_quantise_row(const uint16_t *xr, const float *m, int64_t D, fl
         row_scales[k] = sc;
         float dk = e4m3_decode(sc);
         float inv = dk == 0.0f ? 0.0f : rho_g / dk;
+        if (inv > FLT_MAX) inv = FLT_MAX;
         for (int b = 0; b < B; ++b) {
             float q = bf16_to_f32(xr[k * B + b]) * inv;
             put_code(row_codes, k * B + b, e2m1_encode(q), REF_ELEM_E2M1);
@@ -480,7 +476,7 @@ int rmsnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, float eps, f
             m[k] = mk;
         }
         float r = (float)sqrt(ss / (double)D + (double)eps);
-        float rho = r == 0.0f ? 0.0f : 1.0f / r;
+        float rho = recip_sat(r);
         nvfp4_quantise_row(xr, m, D, rho, global_scale, codes_packed + t * (D / 2), scales_e4m3 + t * K);
         if (rms_out) rms_out[t] = r;
     }
@@ -494,30 +490,48 @@ int rmsnorm_nvfp4_ref(const uint16_t *x_bf16, int64_t T, int64_t D, float eps, f
 /*       dgamma_j = sum_t (x_tj / r_t) g_tj                                    */
 /*       h = g * gamma ; delta_t = (1/D) sum_d h_td x_td                       */
 /*       dX_td = h_td / r_t - x_td * delta_t / r_t^3                           */
+/*     A row whose saved r is 0 is a row of zeros (r~ = 0 only when every      */
+/*     block absmax is 0), for which the forward emitted zeros whatever rho    */
+/*     was: 1/r is taken as 0 there, so the row contributes nothing to dgamma  */
+/*     and gets dX = 0 [reading: the forward's "zero denominator -> rho = 0"]. */
 /* ------------------------------------------------------------------------- */
 int mxnorm_bwd_ref(const uint16_t *x_bf16, const uint16_t *g_bf16, const uint16_t *gain_bf16,
                    const float *rms, int64_t T, int64_t D, double *dx, double *dgain)
 {
     if (T < 0 || D <= 0) return 1;
-    if (dgain) for (int64_t d = 0; d < D; ++d) dgain[d] = 0.0;
-    /* rows in order; the column sum is not parallelised so that it stays a plain loop */
-    for (int64_t t = 0; t < T; ++t) {
-        const uint16_t *xr = x_bf16 + t * D, *gr = g_bf16 + t * D;
-        double r = (double)rms[t];
-        double dot = 0.0;
-        for (int64_t d = 0; d < D; ++d) {
-            double gam = gain_bf16 ? (double)bf16_to_f32(gain_bf16[d]) : 1.0;
-            double h = (double)bf16_to_f32(gr[d]) * gam;
-            dot += h * (double)bf16_to_f32(xr[d]);
+    /* dX: rows are independent */
+    if (dx) {
+#pragma omp parallel for schedule(static)
+        for (int64_t t = 0; t < T; ++t) {
+            const uint16_t *xr = x_bf16 + t * D, *gr = g_bf16 + t * D;
+            double r = (double)rms[t];
+            if (r == 0.0) {   /* zero row: see the note above */
+                for (int64_t d = 0; d < D; ++d) dx[t * D + d] = 0.0;
+                continue;
+            }
+            double dot = 0.0;
+            for (int64_t d = 0; d < D; ++d) {
+                double gam = gain_bf16 ? (double)bf16_to_f32(gain_bf16[d]) : 1.0;
+                double h = (double)bf16_to_f32(gr[d]) * gam;
+                dot += h * (double)bf16_to_f32(xr[d]);
+            }
+            double delta = dot / (double)D;
+            for (int64_t d = 0; d < D; ++d) {
+                double x = (double)bf16_to_f32(xr[d]);
+                double gam = gain_bf16 ? (double)bf16_to_f32(gain_bf16[d]) : 1.0;
+                double h = (double)bf16_to_f32(gr[d]) * gam;
+                dx[t * D + d] = h / r - x * delta / (r * r * r);
+            }
         }
-        double delta = dot / (double)D;
-        for (int64_t d = 0; d < D; ++d) {
-            double x = (double)bf16_to_f32(xr[d]);
-            double g = (double)bf16_to_f32(gr[d]);
-            double gam = gain_bf16 ? (double)bf16_to_f32(gain_bf16[d]) : 1.0;
-            double h = g * gam;
-            if (dx) dx[t * D + d] = h / r - x * delta / (r * r * r);
-            if (dgain) dgain[d] += (x / r) * g;
+    }
+    /* dgamma: the column sum over the rows, in row order, kept a plain serial loop */
+    if (dgain) {
+        for (int64_t d = 0; d < D; ++d) dgain[d] = 0.0;
+        for (int64_t t = 0; t < T; ++t) {
+            double r = (double)rms[t];
+            if (r == 0.0) continue;
+            for (int64_t d = 0; d < D; ++d)
+                dgain[d] += ((double)bf16_to_f32(x_bf16[t * D + d]) / r) * (double)bf16_to_f32(g_bf16[t * D + d]);
         }
     }
     return 0;
@@ -612,6 +626,14 @@ static double postround_estimate(double xbar, const double *nodes, const double 
 
 double mxn_ref_postround_f(double sigma, int B) { return postround_f(sigma, B); }
 double mxn_ref_postround_f_inverse(double x, int B) { return postround_f_inverse(x, B); }
+/* the table-based estimates r~ = f^-1(xbar[i]) exactly as mxnorm_postround_ref evaluates them, before the rounding
+ * to binary32 (the table is built once per call) */
+void mxn_ref_postround_estimate(const double *xbar, int64_t n, int B, double *out)
+{
+    double nodes[POSTROUND_A + 1], values[POSTROUND_A + 1];
+    postround_table(B, nodes, values);
+    for (int64_t i = 0; i < n; ++i) out[i] = postround_estimate(xbar[i], nodes, values);
+}
 
 int mxnorm_postround_ref(const uint16_t *x_bf16, int64_t T, int64_t D, int B, float eps, int mode,
                          uint8_t *codes, uint8_t *scales, float *rms_est_out)
@@ -635,7 +657,7 @@ int mxnorm_postround_ref(const uint16_t *x_bf16, int64_t T, int64_t D, int B, fl
         }
         float rt = (float)postround_estimate(s / (double)K, nodes, values);
         float den = rt + eps;
-        float rho = den == 0.0f ? 0.0f : 1.0f / den;
+        float rho = recip_sat(den);
         for (int64_t d = 0; d < D; ++d) y[d] = bf16_to_f32(xr[d]) * rho;
         quantise_row(y, D, B, mode, REF_ELEM_E4M3, codes + t * D, scales + t * K);
         if (rms_est_out) rms_est_out[t] = rt;
@@ -668,7 +690,7 @@ int mx_cast_transposed_ref(const uint16_t *x_bf16, const float *rms_or_null, int
                 float rho = 1.0f;
                 if (rms_or_null) {
                     float den = rms_or_null[t] + eps;
-                    rho = den == 0.0f ? 0.0f : 1.0f / den;
+                    rho = recip_sat(den);
                 }
                 y[b] = bf16_to_f32(x_bf16[t * D + d]) * rho;
                 float a = fabsf(y[b]);
@@ -708,7 +730,6 @@ float   mxn_ref_e4m3_decode(uint8_t c) { return e4m3_decode(c); }
 uint8_t mxn_ref_e2m1_encode(float q) { return e2m1_encode(q); }
 uint8_t mxn_ref_e5m2_encode(float q) { return e5m2_encode(q); }
 uint8_t mxn_ref_e8m0_scale(float a, int mode, int elem) { return e8m0_scale(a, mode, elem); }
-uint16_t mxn_ref_f64_to_bf16(double v) { return f64_to_bf16(v); }
 
 int mxn_ref_num_threads(void)
 {
