@@ -49,7 +49,8 @@
  *    block absmaxes exact; row statistic accumulated in binary64 and rounded once
  *    to binary32; every element-wise product one IEEE binary32 operation; E8M0
  *    scales by exact exponent tests; element codes round-to-nearest-even,
- *    saturating.
+ *    saturating.  Normalisation factors 1/(r + eps) are 0 for a zero denominator (a row of zeros
+ *    stays zero) and saturate at the largest finite binary32 instead of overflowing.
  */
 #ifndef MXNORM_H_
 #define MXNORM_H_
@@ -69,7 +70,7 @@ typedef enum {
     MXN_ERR_ENUM = 4,      /* unknown rounding mode / layout */
     MXN_ERR_WORKSPACE = 5, /* workspace NULL or smaller than the query says */
     MXN_ERR_CUDA = 6,      /* the CUDA runtime reported an error at launch */
-    MXN_ERR_TIMEOUT = 7,   /* reserved: a bounded device-side wait ran out */
+    MXN_ERR_TIMEOUT = 7,   /* a bounded device-side wait ran out (reported by mxn_device_timeouts) */
     MXN_ERR_TOO_LARGE = 8  /* the problem needs more built-in scratch than the library holds */
 } mxn_status;
 
@@ -90,11 +91,20 @@ size_t mxn_scale_bytes(int64_t T, int64_t K, mxn_scale_layout layout);
 
 const char* mxn_status_string(mxn_status s);
 
-/* Diagnostics: the kernels that wait on asynchronous copies bound every wait; a wait that runs out
- * makes the warp stop and bumps a device-side counter instead of hanging.  This call synchronises the
- * device, stores the number of such events since the library was loaded into *count_out and returns
- * MXN_ERR_TIMEOUT when it is non-zero (outputs of the affected launch are incomplete), else MXN_OK. */
+/* Diagnostics: the one kernel that waits on asynchronous copies (the backward, which feeds its rows through a ring of
+ * shared-memory stages filled by the bulk-copy engine) bounds every wait.  A wait that runs out makes its thread block
+ * stop and bumps a device-side counter instead of hanging: the block requests no further copies, gives the copies it
+ * had already requested a second, shorter bounded wait, writes zeros for its share of the dgain partial sums and
+ * returns.  After such an event the dx rows that block had not reached yet are unwritten and dgain lacks that block's
+ * rows: the outputs of the affected launch are incomplete and must be discarded.
+ *   mxn_device_timeouts synchronises the device, stores the number of such events since the library was loaded (or
+ *   since the last reset) into *count_out and returns MXN_ERR_TIMEOUT when it is non-zero, else MXN_OK.
+ *   mxn_device_timeouts_reset synchronises the device and sets the counter back to 0.
+ *   mxn_selftest_bounded_wait (a test utility) enqueues one warp that waits `polls` times (1..65536) on a barrier
+ *   nobody completes: the wait must run out, be counted exactly once, and the kernel must return normally. */
 mxn_status mxn_device_timeouts(unsigned int* count_out);
+mxn_status mxn_device_timeouts_reset(void);
+mxn_status mxn_selftest_bounded_wait(unsigned int polls, void* cuda_stream);
 
 /* Diagnostics: the NVFP4 kernels replace the IEEE divisions by 6 and by an E4M3 scale with a multiply and two
  * fused multiply-adds that give the same correctly rounded quotient.  This call re-checks that claim on the
@@ -207,7 +217,9 @@ mxn_status mxnorm_mxfp4_fwd(const void* x_bf16, int64_t T, int64_t D, int block,
  *   rms_or_null is NULL (e.g. for the upstream gradient).  Blocks are 32 consecutive tokens of one column;
  *   S and codes as in mx_cast.  Outputs are laid out transposed: codes_t_u8 [D, T] (32-byte aligned),
  *   scales_t_u8 [D, T/32] row-major or tiled with D as the row index (mxn_scale_bytes(D, T/32, layout)).
- *   Requires T % 32 == 0 and D % 4 == 0; x 8-byte aligned. */
+ *   Requires T % 32 == 0 and D % 4 == 0; x 8-byte aligned.  The fast kernel (rows staged in shared memory with
+ *   16-byte copies, output written in whole 128-byte lines) runs when D % 8 == 0 and x is 16-byte aligned; any
+ *   other valid input takes a slower register-only kernel with 8-byte loads. */
 mxn_status mx_cast_transposed(const void* x_bf16, const float* rms_or_null, int64_t T, int64_t D, float eps,
                               void* codes_t_u8, void* scales_t_u8,
                               mxn_round round, mxn_scale_layout layout, void* cuda_stream);
@@ -228,6 +240,8 @@ mxn_status mx_cast_transposed_e5m2(const void* x_bf16, int64_t T, int64_t D,
  *   h = grad_out * gain; delta_t = mean_d(h * x);
  *   dx = h / r - x * delta / r^3        -> dx [T,D], bf16 (dx_is_fp32 == 0) or fp32;
  *   dgain_j = sum_t (x_tj / r_t) * grad_out_tj -> dgain_f32_or_null [D] fp32.
+ *   A row with r_t == 0 (a row of zeros, e.g. a padding token: the forward saved r~ = 0 and emitted zeros) gets
+ *   dx = 0 and adds nothing to dgain.
  *   Row sums in binary32; the column sum is a deterministic two-stage reduction through
  *   `workspace` (device memory, >= mxnorm_bwd_workspace_bytes(T, D) bytes, 16-byte aligned;
  *   contents on entry irrelevant, clobbered on exit; may be NULL when dgain is NULL). */
@@ -268,7 +282,10 @@ size_t mxnorm_bwd_noalloc_max_scratch_bytes(void);
  *   non-blocking streams (created on the first call on each device - make that call outside any
  *   stream capture), ordered after prior work on `cuda_stream` and joined back into it.
  *   The call returns once everything is enqueued; the outputs are valid after `cuda_stream` is
- *   synchronised.  No device memory is allocated. */
+ *   synchronised.  No device memory is allocated.  Calls on one device share the internal streams: they are
+ *   serialised by a lock while they enqueue (thread-safe, but two host threads do not overlap their pipelines).
+ *   If a step fails after work has been enqueued, the caller's stream is still joined with the internal streams
+ *   before the error is returned, so buffers may be reused once `cuda_stream` has been synchronised. */
 mxn_status mxnorm_fwd_host(const void* x_host_bf16, int64_t T, int64_t D, int block, int p, float coef_or_0,
                            float eps, void* codes_host, void* scales_host, float* rms_est_host_or_null,
                            mxn_round round, mxn_scale_layout layout,

@@ -21,7 +21,7 @@ OK = 0
 EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd",
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
-           "mxn_device_timeouts", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
+           "mxn_device_timeouts", "mxn_device_timeouts_reset", "mxn_selftest_bounded_wait", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
            "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
            "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
            "mxnorm_add_fwd", "mx_cast_nvfp4")
@@ -40,6 +40,10 @@ lib.mxn_status_string.argtypes = [_i32]
 lib.mxn_status_string.restype = ctypes.c_char_p
 lib.mxn_device_timeouts.argtypes = [ctypes.POINTER(ctypes.c_uint)]
 lib.mxn_device_timeouts.restype = _i32
+lib.mxn_device_timeouts_reset.argtypes = []
+lib.mxn_device_timeouts_reset.restype = _i32
+lib.mxn_selftest_bounded_wait.argtypes = [ctypes.c_uint, _vp]
+lib.mxn_selftest_bounded_wait.restype = _i32
 lib.mxn_selftest_division.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
 lib.mxn_selftest_division.restype = _i32
 lib.mx_cast.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _i32, _vp]
@@ -110,6 +114,16 @@ def device_timeouts() -> int:
     if st not in (OK, 7):
         raise MXNormError(st, "mxn_device_timeouts")
     return int(n.value)
+
+
+def device_timeouts_reset() -> None:
+    """Synchronises the device and sets the count of run-out waits back to 0."""
+    _check(lib.mxn_device_timeouts_reset(), "mxn_device_timeouts_reset")
+
+
+def selftest_bounded_wait(polls: int = 2000, stream=None) -> None:
+    """Enqueues one warp whose bounded wait (on a barrier nobody completes) must run out after `polls` polls."""
+    _check(lib.mxn_selftest_bounded_wait(polls, _stream(stream)), "mxn_selftest_bounded_wait")
 
 
 def selftest_division() -> int:

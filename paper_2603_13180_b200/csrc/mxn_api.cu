@@ -105,13 +105,21 @@ const char* mxn_status_string(mxn_status s)
 
 mxn_status mxn_device_timeouts(unsigned int* count_out)
 {
-    unsigned int n = 0, nb = 0;
-    if (cudaDeviceSynchronize() != cudaSuccess || mxn::read_timeouts(&n) != cudaSuccess ||
-        mxn::read_timeouts_bwd(&nb) != cudaSuccess)
-        return MXN_ERR_CUDA;
-    n += nb;
+    unsigned int n = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess || mxn::read_timeouts(&n) != cudaSuccess) return MXN_ERR_CUDA;
     if (count_out != nullptr) *count_out = n;
     return n == 0 ? MXN_OK : MXN_ERR_TIMEOUT;
+}
+
+mxn_status mxn_device_timeouts_reset(void)
+{
+    return cudaDeviceSynchronize() == cudaSuccess && mxn::reset_timeouts() == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
+}
+
+mxn_status mxn_selftest_bounded_wait(unsigned int polls, void* cuda_stream)
+{
+    if (polls == 0 || polls > (1u << 16)) return MXN_ERR_SHAPE;
+    return mxn::selftest_bounded_wait(polls, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXN_OK : MXN_ERR_CUDA;
 }
 
 mxn_status mxn_selftest_division(unsigned long long* mismatches_out)
@@ -340,11 +348,11 @@ constexpr int kMaxDevices = 64;
 HostPipe g_pipes[kMaxDevices];
 std::mutex g_pipes_mutex;
 
+// call with g_pipes_mutex held
 HostPipe* host_pipe()
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    std::lock_guard<std::mutex> lock(g_pipes_mutex);
     HostPipe& hp = g_pipes[dev];
     if (!hp.ready) {
         if (cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess ||
@@ -385,6 +393,8 @@ mxn_status mxnorm_fwd_host(const void* x_host_bf16, int64_t T, int64_t D, int bl
     if (workspace == nullptr || workspace_bytes < mxnorm_fwd_host_workspace_bytes(T, D, block, layout))
         return MXN_ERR_WORKSPACE;
     if (misaligned(workspace, 256)) return MXN_ERR_ALIGN;
+    // the internal streams and events of a device are shared by every call on it: one call enqueues at a time
+    std::lock_guard<std::mutex> pipe_lock(g_pipes_mutex);
     HostPipe* hp = host_pipe();
     if (hp == nullptr) return MXN_ERR_CUDA;
     cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
@@ -400,9 +410,10 @@ mxn_status mxnorm_fwd_host(const void* x_host_bf16, int64_t T, int64_t D, int bl
     uint8_t* hcodes = static_cast<uint8_t*>(codes_host);
     uint8_t* hscales = static_cast<uint8_t*>(scales_host);
 
-    bool ok = cudaEventRecord(hp->fork, user) == cudaSuccess &&
-              cudaStreamWaitEvent(hp->in, hp->fork, 0) == cudaSuccess &&
+    if (cudaEventRecord(hp->fork, user) != cudaSuccess) return MXN_ERR_CUDA;   // nothing forked yet
+    bool ok = cudaStreamWaitEvent(hp->in, hp->fork, 0) == cudaSuccess &&
               cudaStreamWaitEvent(hp->out, hp->fork, 0) == cudaSuccess;
+    mxn_status failed = MXN_OK;
     const bool tiled = layout == MXN_SCALES_SWIZZLE_128x4;
     const int64_t tiles_per_row = (K + 3) / 4;
     for (int64_t r0 = 0; ok && r0 < T; r0 += kHostChunkRows) {
@@ -416,15 +427,23 @@ mxn_status mxnorm_fwd_host(const void* x_host_bf16, int64_t T, int64_t D, int bl
         const size_t slen = tiled ? (size_t)((rows + 127) / 128) * tiles_per_row * 512 : (size_t)rows * K;
         mxn_status st = run_fwd(mxn::STAT_MX, false, dx + r0 * D, nullptr, rows, D, block, p, coef_or_0, eps, 1.0f,
                                 dcodes + r0 * D, dscales + soff, drms + r0, round, layout, hp->out);
-        if (st != MXN_OK) return st;
+        if (st != MXN_OK) {   // leave through the join below: the chunks already enqueued must stay ordered
+            failed = st;
+            break;
+        }
         ok = cudaMemcpyAsync(hcodes + r0 * D, dcodes + r0 * D, (size_t)rows * D, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
              cudaMemcpyAsync(hscales + soff, dscales + soff, slen, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
         if (ok && rms_est_host_or_null != nullptr)
             ok = cudaMemcpyAsync(rms_est_host_or_null + r0, drms + r0, (size_t)rows * 4, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
     }
-    ok = ok && cudaEventRecord(hp->join, hp->out) == cudaSuccess &&
-         cudaStreamWaitEvent(user, hp->join, 0) == cudaSuccess;
-    return ok ? MXN_OK : MXN_ERR_CUDA;
+    // Join on every path that forked: the caller's stream waits for both internal streams, so whatever was enqueued
+    // (copies into the caller's buffers included) is ordered before anything the caller enqueues next.
+    const bool joined = cudaEventRecord(hp->copied, hp->in) == cudaSuccess &&
+                        cudaStreamWaitEvent(hp->out, hp->copied, 0) == cudaSuccess &&
+                        cudaEventRecord(hp->join, hp->out) == cudaSuccess &&
+                        cudaStreamWaitEvent(user, hp->join, 0) == cudaSuccess;
+    if (failed != MXN_OK) return failed;
+    return ok && joined ? MXN_OK : MXN_ERR_CUDA;
 }
 
 }  // extern "C"

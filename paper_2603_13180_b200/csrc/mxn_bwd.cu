@@ -51,10 +51,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// false when the barrier did not complete within the spin budget (of the order of a second)
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// false when the barrier did not complete within `limit` polls (the default is of the order of a second)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = 1u << 20)
 {
-    for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+    for (uint32_t spin = 0; spin < limit; ++spin)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -150,7 +150,9 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
                 gw[v] = make_uint4(0, 0, 0, 0);
             }
         }
-        const float inv_r = __fdiv_rn(1.0f, r_row);
+        // a saved r of 0 marks a row of zeros (the forward emitted zeros for it): 1/r is taken as 0, so the row adds
+        // nothing to dgamma and gets dX = 0 instead of 0 * inf = NaN
+        const float inv_r = r_row == 0.0f ? 0.0f : __fdiv_rn(1.0f, r_row);
 
         // One pass over the thread's elements with  gi = g/r,  t = gi*gamma (= h/r):
         //   dgamma += x*gi ;  dot += t*x  (= sum_d h x / r) ;  later  dX = t - x * (dot/(D r^2)).
@@ -178,7 +180,22 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
         if (lane == 0) red[it & 1][warp] = dot;
         __syncthreads();   // row dot complete; every thread has read its part of the stage
         if (abort_flag) {
-            if (tid == 0) atomicAdd(&g_bwd_timeouts, 1u);
+            // A wait ran out: the CTA requests no further copies and stops.  Copies already requested into the other
+            // stages may still be in flight; one thread gives each of them a (shorter) bounded wait so that none lands
+            // after this CTA's shared memory has been handed to another CTA, while the rest zero this CTA's row of
+            // partial sums so that the column sum adds nothing stale.  dX rows from `row` on are left unwritten.
+            if (DGAIN) {
+                float* prow = P.partial + (int64_t)blockIdx.x * P.D;
+                for (int i = tid; i < P.D; i += n) prow[i] = 0.0f;
+            }
+            if (tid == 0) {
+                for (int j = 0; j < stages; ++j) {
+                    const uint32_t itj = it + (uint32_t)j;
+                    if (row + (int64_t)j * stride < P.T)
+                        (void)mbar_wait_bounded(bar0 + 8 * (itj % (uint32_t)stages), (itj / (uint32_t)stages) & 1u, 1u << 16);
+                }
+                atomicAdd(&g_bwd_timeouts, 1u);
+            }
             return;
         }
         if (tid == 0) {
@@ -352,9 +369,33 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     return e;
 }
 
-cudaError_t read_timeouts_bwd(unsigned int* out)
+cudaError_t read_timeouts(unsigned int* out)
 {
     return cudaMemcpyFromSymbol(out, g_bwd_timeouts, sizeof(unsigned int));
+}
+cudaError_t reset_timeouts()
+{
+    const unsigned int zero = 0;
+    return cudaMemcpyToSymbol(g_bwd_timeouts, &zero, sizeof(unsigned int));
+}
+
+// One warp waits, with the given number of polls, on an mbarrier that expects a transfer nobody issues: the wait
+// must run out, be counted, and the kernel must return normally.
+__global__ void __launch_bounds__(32) selftest_bounded_wait_kernel(uint32_t polls)
+{
+    __shared__ uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0 && !mbar_wait_bounded(b, 0, polls)) atomicAdd(&g_bwd_timeouts, 1u);
+}
+cudaError_t selftest_bounded_wait(unsigned int polls, cudaStream_t stream)
+{
+    selftest_bounded_wait_kernel<<<1, 32, 0, stream>>>(polls);
+    return cudaGetLastError();
 }
 
 }  // namespace mxn

@@ -192,6 +192,15 @@ __device__ __forceinline__ bool is_normal_f32(float f)
     return E != 0u && E != 255u;
 }
 
+// ---- normalisation factor ---------------------------------------------------------------------------
+// rho = 1/den as one IEEE binary32 division; 0 for a zero denominator (a zero row stays zero) and the largest finite
+// binary32 where the quotient would overflow (den < 2^-128: rows of subnormal magnitude), so that no 0 * inf = NaN can
+// arise from finite input.
+__device__ __forceinline__ float recip_sat(float den)
+{
+    return den == 0.0f ? 0.0f : fminf(__fdiv_rn(1.0f, den), 3.402823466e+38f);
+}
+
 // ---- programmatic dependent launch ----------------------------------------------------------------
 // Every kernel of the library is launched with programmatic stream serialisation and starts with this
 // prologue: wait until the preceding kernel of the stream has completed and its writes are visible

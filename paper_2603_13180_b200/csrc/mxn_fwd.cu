@@ -447,26 +447,50 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
 }
 
 // ---- host side of the post-round estimator: f, its inverse and the table --------------------------
-// f(sigma) = E[max_i 2^floor(log2 |X_i|)] for B i.i.d. N(0, sigma^2) values
-//          = sum_j 2^j (P(2^(j+1)) - P(2^j)),  P(t) = erf(t / (sigma sqrt 2))^B.
+// f(sigma) = E[Y], Y = 2^floor(log2 max_i |X_i|) for B i.i.d. N(0, sigma^2) values.  Y only takes powers of two, so
+// the expectation is summed over the levels it exceeds:
+//     E[Y] = sum_j (2^j - 2^(j-1)) P(Y >= 2^j) = sum_j 2^(j-1) P(max_i |X_i| >= 2^j),
+//     P(max >= t) = 1 - erf(u)^B = -expm1(B log1p(-erfc(u))),  u = t / (sigma sqrt 2).
+// Levels far below sigma are exceeded with probability 1 to the last bit: their geometric tail is added in closed form.
+static double pr_prob_max_at_least(double t, double sigma, int B)
+{
+    const double u = t / (sigma * 1.4142135623730951);
+    return -std::expm1((double)B * std::log1p(-std::erfc(u)));
+}
 static double pr_expected_rounded_max(double sigma, int B)
 {
-    const double inv = 1.0 / (sigma * std::sqrt(2.0));
-    const int centre = (int)std::floor(std::log2(sigma));
-    double total = 0.0, below = std::pow(std::erf(std::ldexp(1.0, centre - 64) * inv), B);
-    for (int j = centre - 64; j <= centre + 6; ++j) {
-        const double above = std::pow(std::erf(std::ldexp(1.0, j + 1) * inv), B);
-        total += std::ldexp(1.0, j) * (above - below);
-        below = above;
+    int e;
+    (void)std::frexp(sigma, &e);                 // sigma in [2^(e-1), 2^e)
+    const int lowest = e - 14;                   // 2^lowest < sigma 2^-12: erf(u)^B < 2^-160, the probability is exactly 1
+    double total = std::ldexp(1.0, lowest - 1);  // sum over j < lowest of 2^(j-1)
+    for (int j = lowest; j <= e + 8; ++j) {      // beyond 2^8 sigma the probability is below 1e-300
+        const double pj = pr_prob_max_at_least(std::ldexp(1.0, j), sigma, B);
+        if (pj == 0.0) break;
+        total += std::ldexp(pj, j - 1);
     }
     return total;
 }
+// f is increasing and sigma/2 < f(sigma) < 4 sigma for the supported block sizes: a bracketing secant iteration
+// (regula falsi with the Illinois modification) from that bracket
 static double pr_invert(double x, int B)
 {
-    double a = x / 8.0, b = x * 4.0;   // f(sigma) lies between sigma/2 and 4 sigma for these block sizes
-    for (int it = 0; it < 200; ++it) {
-        const double mid = 0.5 * (a + b);
-        (pr_expected_rounded_max(mid, B) < x ? a : b) = mid;
+    double a = x / 8.0, b = x * 4.0;
+    double fa = pr_expected_rounded_max(a, B) - x, fb = pr_expected_rounded_max(b, B) - x;
+    int side = 0;
+    for (int it = 0; it < 200 && b - a > 4e-16 * b; ++it) {
+        double c = (a * fb - b * fa) / (fb - fa);
+        if (!(c > a && c < b)) c = 0.5 * (a + b);
+        const double fc = pr_expected_rounded_max(c, B) - x;
+        if (fc == 0.0) return c;
+        if (fc < 0.0) {
+            a = c; fa = fc;
+            if (side == -1) fb *= 0.5;
+            side = -1;
+        } else {
+            b = c; fb = fc;
+            if (side == 1) fa *= 0.5;
+            side = 1;
+        }
     }
     return 0.5 * (a + b);
 }
@@ -534,14 +558,6 @@ cudaError_t selftest_division(unsigned long long* mismatches_host)
     if (e == cudaSuccess) e = cudaMemcpy(mismatches_host, dev, sizeof(unsigned long long), cudaMemcpyDeviceToHost);
     cudaFree(dev);
     return e;
-}
-
-// number of bounded device-side waits that ran out since the library was loaded (synchronises);
-// no kernel of this build waits on anything, so the counter stays 0
-__device__ unsigned int g_timeouts = 0;
-cudaError_t read_timeouts(unsigned int* out)
-{
-    return cudaMemcpyFromSymbol(out, g_timeouts, sizeof(unsigned int));
 }
 
 }  // namespace mxn

@@ -32,7 +32,6 @@ struct FwdParams {
 
 bool fwd_shape_supported(int64_t D, int B);
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
-cudaError_t read_timeouts(unsigned int* out);
 cudaError_t selftest_division(unsigned long long* mismatches_host);
 cudaError_t postround_prepare(int B);   // uploads the f^-1 table for block size B to the current device (once)
 
@@ -54,8 +53,6 @@ struct BwdParams {
     const uint16_t* x;      // bf16 [T, D]
     const uint16_t* g;      // bf16 [T, D]
     const uint16_t* gain;   // bf16 [D] or nullptr
-    const uint16_t* residual; // bf16 [T, D] or nullptr: added to x before the norm (fused residual add)
-    uint16_t* h_out;        // bf16 [T, D]: x + residual, written when residual is given
     const float* rms;       // [T]
     void* dx;               // bf16 or fp32 [T, D]
     float* dgain;           // [D] or nullptr
@@ -70,6 +67,9 @@ struct BwdParams {
 bool bwd_shape_supported(int64_t D);
 int bwd_parts(int64_t T, int64_t D);
 cudaError_t launch_bwd(BwdParams P, cudaStream_t stream);
-cudaError_t read_timeouts_bwd(unsigned int* out);
+// bounded device-side waits that ran out (the backward's bulk-copy ring is the only code that waits)
+cudaError_t read_timeouts(unsigned int* out);
+cudaError_t reset_timeouts();
+cudaError_t selftest_bounded_wait(unsigned int polls, cudaStream_t stream);
 
 }  // namespace mxn

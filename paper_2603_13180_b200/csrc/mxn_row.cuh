@@ -57,19 +57,17 @@ __device__ __forceinline__ void finish_stat(double s, const FwdParams& P, float&
         double mean = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.K);
         double G = P.p == 2 ? __dsqrt_rn(mean) : mean;
         r = __double2float_rn(__dmul_rn((double)P.coef, G));
-        float den = __fadd_rn(r, P.eps);
-        rho = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
+        rho = recip_sat(__fadd_rn(r, P.eps));
     } else if (STAT == STAT_POSTROUND) {
         // xbar = mean of the power-of-two-rounded block absmaxes; r~ = f^-1(xbar); rho~ = 1 / fl32(r~ + eps)
         const double xbar = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.K);
         r = __double2float_rn(postround_estimate(xbar, P.pr_table));
-        float den = __fadd_rn(r, P.eps);
-        rho = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
+        rho = recip_sat(__fadd_rn(r, P.eps));
     } else if (STAT == STAT_RMS) {
         // r = fl32(sqrt(mean x^2 + eps)); rho = 1 / r
         double ms = P.inv_count != 0.0 ? __dmul_rn(s, P.inv_count) : __ddiv_rn(s, (double)P.D);
         r = __double2float_rn(__dsqrt_rn(__dadd_rn(ms, (double)P.eps)));
-        rho = r == 0.0f ? 0.0f : __fdiv_rn(1.0f, r);
+        rho = recip_sat(r);
     } else {
         r = 1.0f;
         rho = 1.0f;
@@ -128,8 +126,11 @@ __device__ __forceinline__ double block_stats(const uint32_t (&xr)[NPASS][B / 2]
             double md = (double)mc;
             stat = p == 2 ? __fma_rn(md, md, stat) : __dadd_rn(stat, md);   // m^2 is exact in binary64
         }
-        if (STAT == STAT_POSTROUND)   // 2^floor(log2 m): the absmax with its significand cleared (0 stays 0)
-            stat = __dadd_rn(stat, (double)__uint_as_float(__float_as_uint(mc) & 0x7F800000u));
+        if (STAT == STAT_POSTROUND) {   // 2^floor(log2 m): the absmax with its significand cleared (0 stays 0)
+            const uint32_t u = __float_as_uint(mc);
+            const uint32_t p2 = u >= 0x00800000u ? (u & 0x7F800000u) : (u != 0u ? 0x80000000u >> __clz(u) : 0u);   // subnormal: its leading bit
+            stat = __dadd_rn(stat, (double)__uint_as_float(p2));
+        }
         if (STAT == STAT_RMS) {
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
@@ -347,7 +348,7 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
             sc = cvt_e4m3x2(__fmul_rn(div_by_6(a), P.global_scale), 0.0f) & 0xFFu;
             const float d = e4m3_to_f32(sc);
             if (sc >= 8u && rho_g_in_window) inv = div_by_e4m3_normal(rho_g, sc, d);
-            else inv = d == 0.0f ? 0.0f : __fdiv_rn(rho_g, d);
+            else inv = d == 0.0f ? 0.0f : fminf(__fdiv_rn(rho_g, d), 3.402823466e+38f);   // saturates like rho itself
         }
         uint32_t out[2];
         const float2 ii = make_float2(inv, inv);

@@ -53,8 +53,7 @@ __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedPa
     // rho of row t0 + lane
     float rho_l = 1.0f;
     if (P.rms != nullptr) {
-        const float den = __fadd_rn(P.rms[t0 + lane], P.eps);
-        rho_l = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
+        rho_l = recip_sat(__fadd_rn(P.rms[t0 + lane], P.eps));
     }
     uint32_t xr[32][WORDS];
 #pragma unroll
@@ -143,6 +142,9 @@ __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedPa
 #ifndef MXN_TR_MINB
 #define MXN_TR_MINB 12
 #endif
+#ifndef MXN_TO_MINB
+#define MXN_TO_MINB 7   // resident CTAs per SM aimed for (measured at [16384,4096]: 5 -> 35.1 us, 6 -> 32.9, 7 -> 32.0, 8 spills -> 40.1)
+#endif
 constexpr int kTsStages = MXN_TR_TPC > 1 ? 2 : 1;
 #ifndef MXN_TR_COLS
 #define MXN_TR_COLS 128   // columns per CTA tile, 64 per warp (measured at [16384,4096]: 64 -> 36.4 us, 128 -> 34.1, 256 -> 36.0, 512 -> 40.7, 1024 -> 54.2)
@@ -190,8 +192,7 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
             if (tid < 32) {
                 float rho = 1.0f;
                 if (P.rms != nullptr) {
-                    const float den = __fadd_rn(P.rms[t0 + tid], P.eps);
-                    rho = den == 0.0f ? 0.0f : __fdiv_rn(1.0f, den);
+                    rho = recip_sat(__fadd_rn(P.rms[t0 + tid], P.eps));
                 }
                 rho_s[tt & 1][tid] = rho;
             }
@@ -225,6 +226,106 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
     cp_async_wait<0>();
 }
 
+// ---- output-staged variant (D % 8 == 0, x 16-byte aligned) ------------------------------------------
+// A CTA of 4 warps takes a tile of 128 tokens x 64 columns.  The 128 row segments of 128 bytes arrive with 16-byte
+// cp.async copies.  Warp w quantises token block w (32 tokens) of all 64 columns exactly as the kernel above does
+// (a lane owns two adjacent columns), but its 32 code bytes per column go to a shared-memory image of the OUTPUT tile
+// (64 rows of the transposed matrix x 128 tokens); after one barrier the CTA writes that image row by row, eight
+// threads covering the 128 contiguous bytes of one output row - whole lines instead of isolated 32-byte sectors.
+// The 16-byte chunks of an image row are XOR-swizzled with the column pair index so that both the per-lane writes
+// (lane l -> rows 2l, 2l+1) and the row-wise reads are bank-conflict-free.  The four scale bytes of a column (one per
+// token block) leave as one 4-byte store.
+constexpr int kToCols = 64, kToTokens = 128, kToThreads = 128, kToInBytes = kToTokens * kToCols * 2, kToOutBytes = kToCols * kToTokens;
+
+template <bool PAPER, int ELEM, bool ZSPILL>
+__global__ void __launch_bounds__(kToThreads, MXN_TO_MINB) cast_transposed_tile_kernel(const TransposedParams P)
+{
+    extern __shared__ __align__(128) uint8_t tile_raw[];
+    __shared__ __align__(16) float rho_s[4][32];
+    __shared__ __align__(16) uint8_t sb_s[kToCols][4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t in0 = (uint32_t)__cvta_generic_to_shared(tile_raw), out0 = in0 + kToInBytes;
+    const int ctile = blockIdx.x * kToCols;
+    const int64_t tbase = (int64_t)token_tile_index<ZSPILL>() * kToTokens;
+    {   // first-wave CTAs ask for their tile in L2 before the wait for the previous kernel: one 128-byte line per thread
+        const bool first_wave = (uint64_t)token_tile_index<ZSPILL>() * gridDim.x + blockIdx.x < 148u * 9u;
+        if (first_wave && tbase + tid < P.T && ctile < P.D)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(P.x + (tbase + tid) * P.D + ctile) : "memory");
+    }
+    pdl_prologue();
+    if (tbase >= P.T) return;
+    const int nblocks = (int)((P.T - tbase < kToTokens ? P.T - tbase : kToTokens) >> 5);   // token blocks of this tile (T % 32 == 0)
+
+    // 128 rows x 8 chunks of 16 bytes; thread i takes chunk i % 8 of rows i / 8 + 16 k
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int row = (tid >> 3) + 16 * k, c16 = tid & 7;
+        const int col = ctile + c16 * 8;
+        const uint32_t dst = in0 + (uint32_t)row * (kToCols * 2) + (uint32_t)c16 * 16;
+        if (row < nblocks * 32 && col < P.D) cp_async16(dst, P.x + (tbase + row) * P.D + col);
+        else asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" :: "r"(dst), "r"(0u) : "memory");
+    }
+    cp_async_commit();
+    {
+        float rho = 1.0f;
+        if (P.rms != nullptr && tid < nblocks * 32) rho = recip_sat(__fadd_rn(P.rms[tbase + tid], P.eps));
+        rho_s[warp][lane] = rho;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    if (warp < nblocks) {
+        const uint32_t wordaddr = in0 + (uint32_t)(warp * 32) * (kToCols * 2) + (uint32_t)lane * 4;
+        uint32_t xr[32];
+#pragma unroll
+        for (int r = 0; r < 32; ++r) asm volatile("ld.shared.b32 %0, [%1];" : "=r"(xr[r]) : "r"(wordaddr + (uint32_t)r * (kToCols * 2)));
+        uint32_t o0[8], o1[8], sb0, sb1;
+        quantise_column_pair<PAPER, ELEM>(xr, rho_s[warp], P.round, o0, o1, sb0, sb1);
+        // image rows 2*lane and 2*lane+1, bytes [32 warp, 32 warp + 32): chunks 2 warp and 2 warp + 1, swizzled by lane % 8
+        const uint32_t r0 = out0 + (uint32_t)(2 * lane) * kToTokens, sw = (uint32_t)(lane & 7);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t chunk = ((uint32_t)(2 * warp + h) ^ sw) * 16;
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" :: "r"(r0 + chunk), "r"(o0[4 * h]), "r"(o0[4 * h + 1]), "r"(o0[4 * h + 2]), "r"(o0[4 * h + 3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" :: "r"(r0 + kToTokens + chunk), "r"(o1[4 * h]), "r"(o1[4 * h + 1]), "r"(o1[4 * h + 2]), "r"(o1[4 * h + 3]) : "memory");
+        }
+        sb_s[2 * lane][warp] = (uint8_t)sb0;
+        sb_s[2 * lane + 1][warp] = (uint8_t)sb1;
+    }
+    __syncthreads();
+
+    // codes: thread i writes chunk i % 8 of image rows i / 8 + 16 k (eight threads = the 128 contiguous bytes of a row)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int row = (tid >> 3) + 16 * k, j = tid & 7;
+        const int c = ctile + row;
+        if (c < P.D && j < 2 * nblocks) {
+            uint32_t v[4];
+            const uint32_t src = out0 + (uint32_t)row * kToTokens + (((uint32_t)j ^ (uint32_t)((row >> 1) & 7)) * 16);
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(src));
+            st_v4(P.codes + (int64_t)c * P.T + tbase + j * 16, v);
+        }
+    }
+    // scales: thread i < 64 writes the (up to) four scale bytes of column i
+    if (tid < kToCols && ctile + tid < P.D) {
+        const int64_t row = ctile + tid;
+        const int k0 = (int)(tbase >> 5);          // a multiple of 4
+        int64_t off;
+        if (P.layout == MXN_SCALES_ROWMAJOR) {
+            off = row * P.KT + k0;
+        } else {
+            const int rr = (int)(row & 127);
+            off = ((row >> 7) * P.tiles_per_row + (k0 >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4;
+        }
+        const uint32_t w4 = *reinterpret_cast<const uint32_t*>(sb_s[tid]);
+        if (nblocks == 4 && (off & 3) == 0) {
+            *reinterpret_cast<uint32_t*>(P.scales + off) = w4;
+        } else {
+            for (int b = 0; b < nblocks; ++b) P.scales[off + b] = (uint8_t)(w4 >> (8 * b));
+        }
+    }
+}
+
 cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
 {
     P.KT = (int)(P.T / 32);
@@ -241,8 +342,27 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+#ifndef MXN_TR_NO_TILE
+    // 16-byte row chunks need D % 8 == 0 and a 16-byte aligned base (then every row start is 16-byte aligned)
+    if (P.D % 8 == 0 && (reinterpret_cast<uintptr_t>(P.x) & 15) == 0) {
+        const int64_t sx = (P.D + kToCols - 1) / kToCols, sy = (P.T + kToTokens - 1) / kToTokens;
+        if ((sy + kMaxGridY - 1) / kMaxGridY <= 65535) {
+            const bool zs = sy > kMaxGridY;
+            auto kfn = P.elem == ELEM_E5M2 ? (zs ? cast_transposed_tile_kernel<true, 2, true> : cast_transposed_tile_kernel<true, 2, false>)
+                       : P.round == MXN_ROUND_RCEIL_POW2 ? (zs ? cast_transposed_tile_kernel<true, 0, true> : cast_transposed_tile_kernel<true, 0, false>)
+                                                         : (zs ? cast_transposed_tile_kernel<false, 0, true> : cast_transposed_tile_kernel<false, 0, false>);
+            const int smem = kToInBytes + kToOutBytes;
+            const cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e != cudaSuccess) return e;
+            cfg.gridDim = token_tile_grid(sx, sy);
+            cfg.blockDim = dim3(kToThreads);
+            cfg.dynamicSmemBytes = smem;
+            return cudaLaunchKernelEx(&cfg, kfn, P);
+        }
+    }
+#endif
 #ifndef MXN_TR_NO_SMEM
-    if (P.D % 8 == 0) {   // 16-byte row chunks: the shared-memory staged kernel
+    if (P.D % 8 == 0 && (reinterpret_cast<uintptr_t>(P.x) & 15) == 0) {   // 16-byte row chunks: the shared-memory staged kernel
         const int64_t sx = (P.D + kTsCols - 1) / kTsCols, sy = (P.T / 32 + kTsTpc - 1) / kTsTpc;
         if ((sy + kMaxGridY - 1) / kMaxGridY <= 65535) {
             const bool zs = sy > kMaxGridY;

@@ -1,4 +1,6 @@
 """GPU parity of mxnorm_bwd (through the C ABI) against the binary64 oracle."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -92,3 +94,49 @@ def test_backward_with_true_rms_is_orthogonal_to_x(binding, oracle):
     dx, _, _ = run_bwd(binding, x, g, gain, rms, fp32_out=True)
     xv = (x.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     assert np.all(np.abs((dx * xv).sum(-1)) <= 1e-4 * np.abs(dx * xv).sum(-1))
+
+
+def test_backward_with_zero_rows_matches_the_forward_convention(binding, oracle):
+    """Rows of zeros (padding tokens) among normal rows: the forward saves r~ = 0 for them; the backward must give
+    dX = 0 there and a finite dgamma that equals the oracle's (which adds nothing for those rows)."""
+    w = wl.Workload("t", 700, 1024, seed=13, outlier_frac=0.002, has_gain=True, has_grad=True)
+    inp = wl.make_inputs(w)
+    x, g, gain = wl.bits(inp["x"]).copy(), wl.bits(inp["grad"]), wl.bits(inp["gain"])
+    zero_rows = [0, 3, 295, 296, 699]
+    x[zero_rows] = 0
+    x[3, ::2] = 0x8000
+    # the r~ the library's own forward saves
+    xg = wl.from_bits(x).cuda()
+    codes, scales, rms = binding.alloc_outputs(700, 1024)
+    binding.mxnorm_fwd(xg, None, codes, scales, rms, eps=1e-5)
+    torch.cuda.synchronize()
+    r = rms.cpu().numpy()
+    assert np.all(r[zero_rows] == 0) and np.array_equal(r, oracle.mxnorm_ref(x, eps=1e-5)[2])
+    want_dx, want_dg = oracle.mxnorm_bwd_ref(x, g, gain, r)
+    for fp32_out in (True, False):
+        dx, _, dg = run_bwd(binding, x, g, gain, r, fp32_out=fp32_out)
+        assert np.all(np.isfinite(dx)) and np.all(np.isfinite(dg))
+        assert np.all(dx[zero_rows] == 0)
+        scale = np.maximum(np.abs(want_dx).max(-1, keepdims=True), 1e-30)
+        tol = 1e-3 if fp32_out else 2.0 ** -7
+        assert np.all(np.abs(dx - want_dx) <= tol * scale)
+        assert np.all(np.abs(dg - want_dg) <= 1e-3 * np.abs(want_dg).max())
+    assert binding.device_timeouts() == 0
+
+
+def test_a_bounded_wait_that_runs_out_is_counted_and_the_context_stays_usable(binding, oracle):
+    """The only device-side waits of the library are the bounded mbarrier waits of the backward's copy ring.  A test
+    kernel makes such a wait run out (a barrier nobody completes, a few thousand polls): the event must be counted,
+    reported as MXN_ERR_TIMEOUT, resettable, and later launches must work as before."""
+    assert binding.device_timeouts() == 0
+    binding.selftest_bounded_wait(3000)
+    n = ctypes.c_uint(0)
+    st = binding.lib.mxn_device_timeouts(ctypes.byref(n))
+    assert st == 7 and n.value == 1 and "wait" in binding.status_string(st)
+    binding.selftest_bounded_wait(100)
+    assert binding.device_timeouts() == 2
+    binding.device_timeouts_reset()
+    assert binding.device_timeouts() == 0
+    assert binding.lib.mxn_selftest_bounded_wait(0, None) == 2 and binding.lib.mxn_selftest_bounded_wait(1 << 20, None) == 2
+    check(binding, oracle, 65, 2048, seed=3)          # the context is intact: a full backward still matches the oracle
+    assert binding.device_timeouts() == 0

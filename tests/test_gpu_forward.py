@@ -144,13 +144,66 @@ def test_degenerate_rows(binding, oracle):
             # rows 4-7 over/underflow a binary32 sum of squares: outside the baseline's stated domain
             sel = [0, 1, 2, 3]
             gu.assert_within_rounding_of_rho(tuple(a[sel] for a in got), tuple(a[sel] for a in want), 32, "degenerate rms")
-    # NVFP4: row 6 (row scale 2^-126) makes rho~/scale overflow binary32, and 0 * Inf is a NaN whose sign is
-    # not defined: outside the stated domain (row scale within 2^+-100)
-    xs = x[[0, 1, 2, 3, 4, 5, 7]]
-    gu.assert_exact(gu.run_fwd(binding, oracle, "nvfp4", xs), gu.run_ref(oracle, "nvfp4", xs), "degenerate nvfp4")
+    # NVFP4, all rows: for row 6 (row scale 2^-126) rho~ / scale overflows binary32 and saturates at the largest finite
+    # value, so its zeros stay zeros
+    gu.assert_exact(gu.run_fwd(binding, oracle, "nvfp4", x), gu.run_ref(oracle, "nvfp4", x), "degenerate nvfp4")
+    for kind in ("rms_nvfp4", "cast_nvfp4", "mx4", "cast4"):
+        sel = [0, 1, 2, 3] if kind == "rms_nvfp4" else list(range(8))
+        got, want = gu.run_fwd(binding, oracle, kind, x[sel]), gu.run_ref(oracle, kind, x[sel])
+        if kind == "rms_nvfp4":
+            assert np.array_equal(got[0], want[0]) and np.array_equal(got[1], want[1])
+        else:
+            gu.assert_exact(got, want, f"degenerate {kind}")
     # constant-row closed form straight from the GPU: scale 121, code 0x72, r~ = fl32(0.4185)
     codes, scales, r = gu.run_fwd(binding, oracle, "mx", x)
     assert np.all(scales[3] == 121) and np.all(codes[3] == 0x72) and r.view(np.uint32)[3] == 0x3ED645A2
+
+
+def test_subnormal_rows_with_zeros_stay_finite(binding, oracle):
+    """Rows of subnormal magnitude: 1/(r~ + eps) saturates at the largest finite binary32, so zeros stay zeros."""
+    x = np.zeros((6, 128), np.uint16)
+    x[0, ::2] = 0x0001
+    x[1, ::2] = 0x8001
+    x[1, 1::2] = 0x8000
+    x[2, ::2] = 0x0080
+    x[3, ::3] = 0x0003
+    x[4, 5] = 0x0001
+    x[5, :] = 0x0002
+    for kind in ("mx", "nvfp4", "mx4", "postround"):
+        got, want = gu.run_fwd(binding, oracle, kind, x), gu.run_ref(oracle, kind, x)
+        if kind == "postround":
+            assert np.array_equal(got[0], want[0]) and np.array_equal(got[1], want[1])
+        else:
+            gu.assert_exact(got, want, f"subnormal rows {kind}")
+    for block in (16, 64):
+        gu.assert_exact(gu.run_fwd(binding, oracle, "mx", x, block=block), gu.run_ref(oracle, "mx", x, block=block), "subnormal rows")
+    got = gu.run_fwd(binding, oracle, "rms", x)
+    want = gu.run_ref(oracle, "rms", x)
+    assert np.all((got[0][:, 1::2] & 0x7F)[:3] == 0) and not np.any((got[0] & 0x7F) == 0x7F)
+
+
+def test_nvfp4_at_the_edge_of_the_stated_domain(binding, oracle):
+    """Row scales 2^-100 and 2^+100, blocks whose E4M3 scale is subnormal or zero, global scales that push the scale
+    into saturation: every byte must equal the oracle's."""
+    base, _ = rows(48, 512, seed=91)
+    bv = (base.astype(np.uint32) << 16).view(np.float32).copy()
+    bv[:, 16:32] *= np.float32(2.0 ** -5)         # E4M3 scale in its subnormal range
+    bv[:, 32:48] *= np.float32(2.0 ** -12)        # scale rounds to zero: codes +-0
+    bv[:, 48:64] *= np.float32(2.0 ** -9)         # at the bottom of the subnormal range
+    base = wl.f32_to_bf16_bits(bv)
+    want0 = gu.run_ref(oracle, "nvfp4", base)
+    assert np.any((want0[1][:, 1] > 0) & (want0[1][:, 1] < 8)) and np.all(want0[1][:, 2] == 0)
+    for k in (-100, -90, 0, 90, 100):
+        xs = wl.f32_to_bf16_bits(bv * np.float32(2.0 ** k))
+        for p, eps in ((2, 0.0), (1, 0.0)):
+            got = gu.run_fwd(binding, oracle, "nvfp4", xs, p=p, eps=eps)
+            gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", xs, p=p, eps=eps), f"nvfp4 row scale 2^{k}")
+        if k in (-100, 100):
+            assert np.array_equal(got[0], gu.run_ref(oracle, "nvfp4", base, p=1)[0])      # the shift changes no code
+        gu.assert_exact(gu.run_fwd(binding, oracle, "cast_nvfp4", xs), gu.run_ref(oracle, "cast_nvfp4", xs), "mx_cast_nvfp4 at the edge")
+    for gs in (2.0 ** -8, 64.0, 2.0 ** 12):        # tiny scales / scales saturating at 448
+        got = gu.run_fwd(binding, oracle, "nvfp4", base, global_scale=gs)
+        gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", base, global_scale=gs), f"nvfp4 global scale {gs}")
 
 
 @pytest.mark.parametrize("T,D", [(1, 16), (5, 48), (37, 768), (130, 1024), (33, 4096), (5, 8192), (3, 16384), (257, 2048),

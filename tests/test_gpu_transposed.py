@@ -38,7 +38,8 @@ def run(binding, oracle, x_bits, rms, eps=0.0, round=0, layout=0):
     return codes.cpu().numpy().reshape(D, T), s_np
 
 
-@pytest.mark.parametrize("T,D", [(32, 4), (64, 128), (96, 160), (160, 132), (256, 4096), (2048, 768), (128, 5120)])
+@pytest.mark.parametrize("T,D", [(32, 4), (64, 128), (96, 160), (160, 132), (256, 4096), (2048, 768), (128, 5120),
+                                 (32, 64), (288, 72), (416, 200), (1024, 1280)])
 def test_transposed_cast_matches_oracle_bit_for_bit(binding, oracle, T, D):
     inp = wl.make_inputs(wl.Workload("t", T, D, seed=T + D, outlier_frac=0.01 if D >= 100 else 0.0))
     x = wl.bits(inp["x"])
@@ -72,6 +73,40 @@ def test_transposed_cast_full_size_with_the_forward_estimate(binding, oracle):
     c, s = run(binding, oracle, g, None)
     wc, ws = oracle.mx_cast_transposed_ref(g)
     assert np.array_equal(s, ws) and np.array_equal(c, wc)
+
+
+def test_transposed_cast_of_an_input_that_is_only_8_byte_aligned(binding, oracle):
+    """A contiguous view whose base address is 8 mod 16 is valid input (the contract asks for 8 bytes): it must take
+    the register kernel with 8-byte loads, not the kernel that stages rows with 16-byte copies."""
+    T, D = 160, 256
+    inp = wl.make_inputs(wl.Workload("t", T, D, seed=77, outlier_frac=0.01))
+    x_bits = wl.bits(inp["x"])
+    buf = torch.zeros(T * D + 4, dtype=torch.bfloat16, device="cuda")
+    assert buf.data_ptr() % 16 == 0
+    x = buf[4:].view(T, D)                                   # base address = 8 mod 16
+    x.copy_(inp["x"])
+    assert x.data_ptr() % 16 == 8 and x.is_contiguous()
+    xv = (x_bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    r_est = (1.03 * np.sqrt((xv ** 2).mean(-1))).astype(np.float32)
+    r = torch.from_numpy(r_est).cuda()
+    for layout in (0, 1):
+        cfull, codes = gu.guarded(D * T)
+        sbytes = binding.scale_bytes(D, T // 32, layout)
+        sfull, scales = gu.guarded(sbytes)
+        binding.mx_cast_transposed(x, r, codes, scales, eps=1e-5, layout=layout)
+        torch.cuda.synchronize()
+        assert gu.guards_intact(cfull, D * T) and gu.guards_intact(sfull, sbytes)
+        wc, ws = oracle.mx_cast_transposed_ref(x_bits, rms=r_est, eps=1e-5)
+        s_np = scales.cpu().numpy()
+        s_np = gu.unswizzle(s_np, D, T // 32, oracle) if layout == 1 else s_np.reshape(D, T // 32)
+        assert np.array_equal(s_np, ws) and np.array_equal(codes.cpu().numpy().reshape(D, T), wc)
+    # the E5M2 variant shares the dispatch
+    cfull, codes = gu.guarded(D * T)
+    sfull, scales = gu.guarded(D * (T // 32))
+    binding.mx_cast_transposed_e5m2(x, codes, scales)
+    torch.cuda.synchronize()
+    wc, ws = oracle.mx_cast_transposed_ref(x_bits, elem=oracle.ELEM_E5M2)
+    assert np.array_equal(scales.cpu().numpy().reshape(D, T // 32), ws) and np.array_equal(codes.cpu().numpy().reshape(D, T), wc)
 
 
 def test_transposed_cast_argument_errors(binding):

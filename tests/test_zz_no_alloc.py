@@ -4,8 +4,9 @@ built into the library, shared by every call on the device.  This file is collec
 if the built-in scratch misbehaves, every other test has already run.
 
 The GPU test calls the new entry point through the C ABI twice in a row, on different inputs, and
-checks each result against the existing mxnorm_bwd (caller-provided workspace) with the tolerance the
-backward tests use; the second call has fewer partial rows than the first, so stale scratch contents
+checks each result against the existing mxnorm_bwd (caller-provided workspace): within the tolerance the
+backward tests use, and - because both entry points launch the same kernels on the same inputs - bit for bit;
+the second call has fewer partial rows than the first, so stale scratch contents
 from the first call would show up in its dgain."""
 import numpy as np
 import pytest
@@ -44,6 +45,7 @@ def _close(dx_a, dg_a, dx_b, dg_b):
     assert np.all(np.isfinite(dx_b)) and np.all(np.isfinite(dg_b))
     assert np.all(np.abs(dx_b - dx_a) <= ROW_TOL * scale)
     assert np.all(np.abs(dg_b - dg_a) <= ROW_TOL * np.abs(dg_a).max())
+    assert np.array_equal(dx_a, dx_b) and np.array_equal(dg_a, dg_b)     # same kernels, same inputs: identical bits
 
 
 @pytest.mark.gpu
