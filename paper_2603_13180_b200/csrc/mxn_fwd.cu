@@ -204,6 +204,177 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
     quantise_store_nvfp4<NPASS, WPR>(xr, m, rho, P, row, w, lane);
 }
 
+// NVFP4 with two blocks per lane and pass (rows of an even number of blocks): see quantise_pair_nvfp4
+template <int NPASS, int WPR, int STAT>
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvfp4_pair_kernel(const FwdParams P)
+{
+    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / WPR, w = warp - group * WPR;
+    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
+    prefetch_row(P.x, row, P, w, lane);
+    pdl_prologue();
+    if (row >= P.T) return;
+
+    uint32_t xr[NPASS][16];
+    float m0[NPASS], m1[NPASS];
+    load_row_direct<32, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
+    double stat = 0.0;
+    float2 ssa = make_float2(0.f, 0.f), ssb = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        uint32_t ma = absmax_bf16x2(xr[i][0], xr[i][1]), mb = absmax_bf16x2(xr[i][8], xr[i][9]);
+#pragma unroll
+        for (int j = 2; j < 8; ++j) {
+            ma = absmax_bf16x2(ma, xr[i][j]);
+            mb = absmax_bf16x2(mb, xr[i][8 + j]);
+        }
+        m0[i] = hmax_abs_to_f32(ma);
+        m1[i] = hmax_abs_to_f32(mb);
+        if (STAT == STAT_MX) {
+            const double d0 = (double)m0[i], d1 = (double)m1[i];
+            stat = P.p == 2 ? __fma_rn(d1, d1, __fma_rn(d0, d0, stat)) : __dadd_rn(__dadd_rn(stat, d0), d1);
+        }
+        if (STAT == STAT_RMS) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+                const float2 a = bf16x2_to_f32x2(xr[i][j]), b = bf16x2_to_f32x2(xr[i][j + 1]);
+                ssa = __ffma2_rn(a, a, ssa);
+                ssb = __ffma2_rn(b, b, ssb);
+            }
+        }
+    }
+    if (STAT == STAT_RMS) {
+        stat = (double)ssa.x + (double)ssa.y + ((double)ssb.x + (double)ssb.y);
+        forget_unpacked<NPASS, 16>(xr);
+    }
+    float r = 1.0f, rho = 1.0f;
+    if (STAT != STAT_NONE) {
+        stat = group_sum<WPR>(stat, group, w, red);
+        finish_stat<STAT>(stat, P, r, rho);
+        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
+    }
+    quantise_store_nvfp4_pair<NPASS, WPR>(xr, m0, m1, rho, P, row, w, lane);
+}
+
+// ---- several short rows per warp ----------------------------------------------------------------------------------
+// One warp, no shared memory: a row spans RSPAN passes of the warp (piece k of a row goes to pass k / 32, lane k % 32) and
+// the warp takes NPASS / RSPAN consecutive rows.  Pieces may be smaller than a block (E = 16 elements, LPB lanes per
+// block), which lets rows of 5 * 2^r blocks fill whole passes of one warp.  The row statistics are independent shuffle
+// reductions, one per row.
+template <int E, int LPB, int NPASS, int RSPAN, int STAT, int FMT>
+__global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_multi_kernel(const FwdParams P)
+{
+    constexpr int W = E / 2, RPW = NPASS / RSPAN;
+    static_assert(NPASS % RSPAN == 0 && (E == 16 || E == 32), "whole rows per warp; 32- or 64-byte pieces");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row0 = ((int64_t)blockIdx.x * MXN_FWD_WARPS + warp) * RPW;
+    if (lane == 0 && blockIdx.x < kFirstWaveCtas && row0 < P.T) {
+        const int64_t nrows = P.T - row0 < RPW ? P.T - row0 : RPW;
+        prefetch_l2_bulk(P.x + row0 * P.D, (uint32_t)(nrows * P.D) * 2u);
+    }
+    pdl_prologue();
+    if (row0 >= P.T) return;
+
+    uint32_t xr[NPASS][W];
+    float m[NPASS];
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        const int64_t row = row0 + i / RSPAN;
+        const int k = (i % RSPAN) * 32 + lane;
+        if (row < P.T && k < P.chunks) {
+            const uint16_t* p = P.x + row * P.D + (int64_t)k * E;
+#pragma unroll
+            for (int v = 0; v < W / 8; ++v) ld_v8(p + v * 16, &xr[i][v * 8]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < W; ++q) xr[i][q] = 0u;
+        }
+    }
+    double stat[RPW];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) stat[r] = 0.0;
+    float2 ssa[RPW], ssb[RPW];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) ssa[r] = ssb[r] = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        uint32_t m2 = absmax_bf16x2(xr[i][0], xr[i][1]);
+#pragma unroll
+        for (int q = 2; q < W; ++q) m2 = absmax_bf16x2(m2, xr[i][q]);
+        m[i] = hmax_abs_to_f32(m2);
+#pragma unroll
+        for (int o = 1; o < LPB; o <<= 1) m[i] = fmaxf(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], o));
+        const float mc = (LPB == 1 || (lane & (LPB - 1)) == 0) ? m[i] : 0.0f;
+        if (STAT == STAT_MX) {
+            const double md = (double)mc;
+            stat[i / RSPAN] = P.p == 2 ? __fma_rn(md, md, stat[i / RSPAN]) : __dadd_rn(stat[i / RSPAN], md);
+        }
+        if (STAT == STAT_RMS) {
+#pragma unroll
+            for (int q = 0; q < W; q += 2) {
+                const float2 a = bf16x2_to_f32x2(xr[i][q]), b = bf16x2_to_f32x2(xr[i][q + 1]);
+                ssa[i / RSPAN] = __ffma2_rn(a, a, ssa[i / RSPAN]);
+                ssb[i / RSPAN] = __ffma2_rn(b, b, ssb[i / RSPAN]);
+            }
+        }
+    }
+    if (STAT == STAT_RMS) forget_unpacked<NPASS, W>(xr);
+    float rho[RPW];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+        rho[r] = 1.0f;
+        if (STAT != STAT_NONE) {
+            if (STAT == STAT_RMS) stat[r] = (double)ssa[r].x + (double)ssa[r].y + ((double)ssb[r].x + (double)ssb[r].y);
+            float rr;
+            finish_stat<STAT>(warp_sum(stat[r]), P, rr, rho[r]);
+            if (P.rms_out != nullptr && lane == 0 && row0 + r < P.T) P.rms_out[row0 + r] = rr;
+        }
+    }
+    const float rcp_sig = FMT == 2 ? kRcpE4M3Significand[lane & 7] : 0.0f;
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        const int64_t row = row0 + i / RSPAN;
+        const int k = (i % RSPAN) * 32 + lane;
+        const bool active = row < P.T && k < P.chunks;
+        const float rh = rho[i / RSPAN];
+        uint32_t sbyte;
+        if constexpr (FMT == 0) {
+            uint32_t out[W / 2];
+            sbyte = quantise_piece_fp8<E, true, 0>(xr[i], m[i], rh, is_normal_f32(rh), active, 0, out);
+            if (active) {
+                uint8_t* cp = P.codes + row * P.D + (int64_t)k * E;
+                if constexpr (E == 16) st_v4(cp, out);
+                else st_v8(cp, out);
+            }
+        } else if constexpr (FMT == 1) {
+            uint32_t out[W / 4];
+            sbyte = quantise_piece_mxfp4<E>(xr[i], m[i], rh, is_normal_f32(rh), active, out);
+            if (active) {
+                uint8_t* cp = P.codes + row * (P.D / 2) + (int64_t)k * (E / 2);
+                if constexpr (E == 16) st_v2(cp, out);
+                else st_v4(cp, out);
+            }
+        } else {
+            uint32_t out[2];
+            const float rho_g = __fmul_rn(rh, P.global_scale);
+            sbyte = quantise_piece_nvfp4(xr[i], m[i], rh, rho_g, in_division_window(rho_g), rcp_sig, P.global_scale, active, out);
+            if (active) st_v2(P.codes + row * (P.D / 2) + (int64_t)k * 8, out);
+        }
+        if (active && (LPB == 1 || (lane & (LPB - 1)) == 0)) {
+            const int kb = k / LPB;
+            int64_t off;
+            if (P.layout == MXN_SCALES_ROWMAJOR) {
+                off = row * P.K + kb;
+            } else {
+                const int rr = (int)(row & 127);
+                off = ((row >> 7) * P.tiles_per_row + (kb >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (kb & 3);
+            }
+            P.scales[off] = (uint8_t)sbyte;
+        }
+    }
+}
+
 // ---- dispatch ---------------------------------------------------------------------------------
 typedef void (*fwd_fn)(const FwdParams);
 
@@ -358,6 +529,47 @@ static fwd_fn pick_nvfp4(int wpr, int npass)
     return nullptr;
 }
 
+// The one-warp kernel with 16-element pieces is used where it measured faster than the row-group kernels: rows of
+// exactly 160 pieces (D = 2560), five passes of one warp instead of three warps x one pass or two warps x four passes
+// ([16384, 2560]: 5.7 -> 5.9 TB/s for blocks of 32, 5.3 -> 6.1 for blocks of 16, NVFP4 4.5 -> 5.1).  Measured and not
+// kept: two rows of 32 pieces per warp (D = 1024: 5.5 -> 5.2 TB/s), three passes of 16-element pieces (D = 1536:
+// 5.8 -> 5.5) and 8-element pieces, four lanes per block (D = 1280: 5.1 -> 3.8, D = 1792: 6.1 -> 4.0).
+static bool use_one_warp_kernel(int64_t D, int B) { return D == 2560 && (B == 16 || B == 32 || B == 64); }
+
+template <int FMT, int STAT>
+static fwd_fn pick_multi(int B)
+{
+    if constexpr (FMT == 2) return fwd_multi_kernel<16, 1, 5, 5, STAT, 2>;
+    else return B == 16 ? fwd_multi_kernel<16, 1, 5, 5, STAT, FMT> : B == 32 ? fwd_multi_kernel<16, 2, 5, 5, STAT, FMT> : fwd_multi_kernel<16, 4, 5, 5, STAT, FMT>;
+}
+template <int FMT>
+static fwd_fn pick_multi_stat(int B, int stat)
+{
+    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B) : pick_multi<FMT, STAT_NONE>(B);
+}
+
+template <int NPASS, int STAT>
+static fwd_fn nvfp4_pair_by_wpr(int wpr)
+{
+    switch (wpr) {
+        case 1: return fwd_nvfp4_pair_kernel<NPASS, 1, STAT>;
+        case 2: return fwd_nvfp4_pair_kernel<NPASS, 2, STAT>;
+        case 3: return fwd_nvfp4_pair_kernel<NPASS, 3, STAT>;
+        case 4: return fwd_nvfp4_pair_kernel<NPASS, 4, STAT>;
+        case 5: return fwd_nvfp4_pair_kernel<NPASS, 5, STAT>;
+        case 6: return fwd_nvfp4_pair_kernel<NPASS, 6, STAT>;
+        case 7: return fwd_nvfp4_pair_kernel<NPASS, 7, STAT>;
+        case 8: return fwd_nvfp4_pair_kernel<NPASS, 8, STAT>;
+        case 16: return fwd_nvfp4_pair_kernel<NPASS, 16, STAT>;
+        default: return nullptr;
+    }
+}
+template <int STAT>
+static fwd_fn pick_nvfp4_pair(int wpr, int npass)
+{
+    return npass == 2 ? nvfp4_pair_by_wpr<2, STAT>(wpr) : npass == 1 ? nvfp4_pair_by_wpr<1, STAT>(wpr) : nullptr;
+}
+
 // Splits the K per-lane pieces of a row (B elements each) over WPR warps x NPASS passes (at most MXN_FWD_MAX_ELEMS
 // elements per lane), choosing among the instantiated kernels by the fraction of idle lanes, with a handicap for
 // splits that leave a lane little work when a row spans several warps (more warps, hence more synchronisation,
@@ -406,12 +618,19 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
     const bool e5m2 = P.elem == ELEM_E5M2;
     const bool add = P.residual != nullptr;
-    const int E = B == 64 ? 32 : B;   // elements per lane and pass; a block of 64 is shared by two lanes
+#ifdef MXN_NVFP4_NO_PAIR
+    const bool nv_pair = false;
+#else
+    // NVFP4 rows of an even number of blocks: a lane owns two adjacent blocks (about a fifth fewer instructions).  Measured
+    // 1-3 % faster than one block per lane up to D = 10240 and 2-10 % slower from D = 12288 on (65536 rows), hence the limit.
+    const bool nv_pair = nvfp4 && P.K % 2 == 0 && P.D < 12288;
+#endif
+    const int E = nv_pair ? 32 : B == 64 ? 32 : B;   // elements per lane and pass; a block of 64 is shared by two lanes
     const bool fine = nvfp4 || (!mxfp4 && !e5m2 && !add && stat != STAT_POSTROUND && P.gain == nullptr &&
                                 P.round == MXN_ROUND_RCEIL_POW2);
     P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
-    P.chunks = P.K * (B / E);
-    if (!plan_row(P.chunks, E, fine, nvfp4, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
+    P.chunks = nv_pair ? P.K / 2 : P.K * (B / E);
+    if (!plan_row(P.chunks, E, fine, nvfp4 && !nv_pair, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
     P.tiles_per_row = (P.K + 3) / 4;
     {
         const int count = stat == STAT_RMS ? P.D : P.K;   // divisor of the row statistic
@@ -421,7 +640,26 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     P.rows_per_cta = rows_per_cta(P.wpr);
     const bool has_gain = P.gain != nullptr;
     fwd_fn fn = nullptr;
-    if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
+    if ((fine || mxfp4) && stat != STAT_POSTROUND && use_one_warp_kernel(P.D, B)) {
+        constexpr int kE = 16, kPasses = 5;
+        fn = nvfp4 ? pick_multi_stat<2>(16, stat) : mxfp4 ? pick_multi_stat<1>(B, stat) : pick_multi_stat<0>(B, stat);
+        P.chunks = (int)(P.D / kE);
+        (void)kPasses;
+        const int64_t ctas = (P.T + MXN_FWD_WARPS - 1) / MXN_FWD_WARPS;
+        if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)ctas);
+        cfg.blockDim = dim3(MXN_FWD_WARPS * kWarp);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, fn, P);
+    }
+    if (nv_pair) fn = stat == STAT_RMS ? pick_nvfp4_pair<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4_pair<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4_pair<STAT_MX>(P.wpr, P.npass);
+    else if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
     else if (add) fn = B == 16 ? pick_add_mx<16, 1>(P.wpr, P.npass) : B == 32 ? pick_add_mx<32, 1>(P.wpr, P.npass) : pick_add_mx<32, 2>(P.wpr, P.npass);
     else if (e5m2) fn = B == 16 ? pick_e5m2<16, 1>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32, 1>(P.wpr, P.npass) : pick_e5m2<32, 2>(P.wpr, P.npass);
     else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16, 1>(stat, P.wpr, P.npass)

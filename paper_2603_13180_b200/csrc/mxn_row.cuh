@@ -171,6 +171,110 @@ __device__ __forceinline__ void scale_addressing(const FwdParams& P, int64_t row
     }
 }
 
+// ---- one piece (B contiguous elements of one lane), given the row's rho ----------------------------------------
+// E4M3 / E5M2 codes with an E8M0 scale, the paper's rounding rule or P.round: returns the scale byte, out[] = the codes.
+// The __all_sync inside makes the choice between the one-product and the two-product form warp-uniform, so every lane
+// of the warp must call this (inactive lanes with zero data).
+template <int B, bool PAPER, int ELEM>
+__device__ __forceinline__ uint32_t quantise_piece_fp8(const uint32_t (&x)[B / 2], float m, float rho, bool rho_normal, bool active,
+                                                       int round, uint32_t (&out)[B / 4])
+{
+    constexpr int W = B / 2;
+    // a = fl32(m * rho) is also the absmax of fl32(x * rho): rounding is monotone
+    const float a = __fmul_rn(m, rho);
+    const uint32_t sb = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(a) : e8m0_scale(a, round);
+    const float inv = inv_scale(sb);
+    // q = fl32(x*rho) * 2^(127-sb).  When neither factor product leaves the normal range the
+    // two roundings collapse into the single product x * (rho * 2^(127-sb)).
+    const float f = __fmul_rn(rho, inv);
+    const bool fast = sb >= 16u && rho_normal && is_normal_f32(f);
+    if (__all_sync(0xFFFFFFFFu, fast || !active)) {
+        const float2 ff = make_float2(f, f);
+#pragma unroll
+        for (int j = 0; j < W; j += 2) {
+            const float2 q0 = mul2(bf16x2_to_f32x2(x[j]), ff), q1 = mul2(bf16x2_to_f32x2(x[j + 1]), ff);
+            out[j / 2] = cvt_fp8x4<ELEM>(q0.x, q0.y, q1.x, q1.y);
+        }
+    } else {
+        const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
+#pragma unroll
+        for (int j = 0; j < W; j += 2) {
+            const float2 q0 = mul2(mul2(bf16x2_to_f32x2(x[j]), rr), ii);
+            const float2 q1 = mul2(mul2(bf16x2_to_f32x2(x[j + 1]), rr), ii);
+            out[j / 2] = cvt_fp8x4<ELEM>(q0.x, q0.y, q1.x, q1.y);
+        }
+    }
+    return sb;
+}
+
+// MXFP4: E2M1 codes two per byte with an E8M0 scale, S = 2^(ceil(log2 a) - 2) (4 = 2^2 is the largest power of two of E2M1)
+template <int B>
+__device__ __forceinline__ uint32_t quantise_piece_mxfp4(const uint32_t (&x)[B / 2], float m, float rho, bool rho_normal, bool active,
+                                                         uint32_t (&out)[B / 8])
+{
+    constexpr int W = B / 2;
+    const float a = __fmul_rn(m, rho);
+    const uint32_t u = __float_as_uint(a), E = u >> 23;
+    uint32_t sb;
+    if (E >= 255u) sb = (u & 0x7FFFFFu) ? 0u : 254u;   // not finite (outside the contract)
+    else sb = (uint32_t)max((int)E + ((u & 0x7FFFFFu) != 0u) - 2, 0);
+    const float inv = inv_scale(sb);
+    const float f = __fmul_rn(rho, inv);
+    const bool fast = sb >= 16u && rho_normal && is_normal_f32(f);   // same argument as for E4M3
+    if (__all_sync(0xFFFFFFFFu, fast || !active)) {
+        const float2 ff = make_float2(f, f);
+#pragma unroll
+        for (int j = 0; j < W; j += 4) {
+            const float2 q0 = mul2(bf16x2_to_f32x2(x[j]), ff), q1 = mul2(bf16x2_to_f32x2(x[j + 1]), ff);
+            const float2 q2 = mul2(bf16x2_to_f32x2(x[j + 2]), ff), q3 = mul2(bf16x2_to_f32x2(x[j + 3]), ff);
+            out[j / 4] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
+        }
+    } else {
+        const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
+#pragma unroll
+        for (int j = 0; j < W; j += 4) {
+            const float2 q0 = mul2(mul2(bf16x2_to_f32x2(x[j]), rr), ii), q1 = mul2(mul2(bf16x2_to_f32x2(x[j + 1]), rr), ii);
+            const float2 q2 = mul2(mul2(bf16x2_to_f32x2(x[j + 2]), rr), ii), q3 = mul2(mul2(bf16x2_to_f32x2(x[j + 3]), rr), ii);
+            out[j / 4] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
+        }
+    }
+    return sb;
+}
+
+// NVFP4: one block of 16 elements: E4M3 block scale = E4M3(fl32(fl32(a/6) * global_scale)), a = fl32(m * rho~);
+// element factor = fl32(rho~ * global_scale) / scale (0 when the scale is 0, saturating).  rho_g = fl32(rho * global_scale);
+// rcp_sig = RN(1/(1+j/8)) for j = lane % 8 (fetched from the lane that holds the needed one with a shuffle: a
+// lane-dependent index into constant memory would be replayed once per distinct index).  Every lane of the warp must call.
+__device__ __forceinline__ uint32_t quantise_piece_nvfp4(const uint32_t (&x)[8], float m, float rho, float rho_g, bool rho_g_in_window,
+                                                         float rcp_sig, float global_scale, bool active, uint32_t (&out)[2])
+{
+    const float a = __fmul_rn(m, rho);
+    // the common case first, without the IEEE division sequences and decided for the whole warp at once:
+    // numerators inside the window of the exact shortcut and a normal E4M3 scale
+    uint32_t sc = cvt_e4m3x2(__fmul_rn(div_by_known(a, 6.0f, 0x1.555556p-3f), global_scale), 0.0f) & 0xFFu;
+    const bool common = in_division_window(a) && sc >= 8u && rho_g_in_window;
+    float inv;
+    if (__all_sync(0xFFFFFFFFu, common || !active)) {
+        const float d = __uint_as_float((sc << 20) + (120u << 23));            // (8+mf) * 2^(ef-10)
+        const float c = __fmul_rn(__shfl_sync(0xFFFFFFFFu, rcp_sig, (int)(sc & 7u)), __uint_as_float((134u - (sc >> 3)) << 23));
+        inv = div_by_known(rho_g, d, c);
+    } else {
+        sc = cvt_e4m3x2(__fmul_rn(div_by_6(a), global_scale), 0.0f) & 0xFFu;
+        const float d = e4m3_to_f32(sc);
+        if (sc >= 8u && rho_g_in_window) inv = div_by_e4m3_normal(rho_g, sc, d);
+        else inv = d == 0.0f ? 0.0f : fminf(__fdiv_rn(rho_g, d), 3.402823466e+38f);   // saturates like rho itself
+    }
+    const float2 ii = make_float2(inv, inv);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t* xw = &x[h * 4];
+        const float2 q0 = mul2(bf16x2_to_f32x2(xw[0]), ii), q1 = mul2(bf16x2_to_f32x2(xw[1]), ii);
+        const float2 q2 = mul2(bf16x2_to_f32x2(xw[2]), ii), q3 = mul2(bf16x2_to_f32x2(xw[3]), ii);
+        out[h] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
+    }
+    return sc;
+}
+
 // phase 2 (E4M3 codes, E8M0 scales): scales, codes and their stores for this lane's blocks.
 // PAPER selects the paper's rounding rule at compile time (the common case); otherwise P.round decides.
 template <int B, int NPASS, int WPR, bool GAIN, bool PAPER, int ELEM = 0, int LPB = 1>
@@ -190,30 +294,7 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
         uint32_t out[W / 2];
         uint32_t sb;
         if (!GAIN) {
-            // a = fl32(m * rho) is also the absmax of fl32(x * rho): rounding is monotone
-            const float a = __fmul_rn(m[i], rho);
-            sb = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(a) : e8m0_scale(a, P.round);
-            const float inv = inv_scale(sb);
-            // q = fl32(x*rho) * 2^(127-sb).  When neither factor product leaves the normal range the
-            // two roundings collapse into the single product x * (rho * 2^(127-sb)).
-            const float f = __fmul_rn(rho, inv);
-            const bool fast = sb >= 16u && rho_normal && is_normal_f32(f);
-            if (__all_sync(0xFFFFFFFFu, fast || !active)) {
-                const float2 ff = make_float2(f, f);
-#pragma unroll
-                for (int j = 0; j < W; j += 2) {
-                    const float2 q0 = mul2(bf16x2_to_f32x2(xr[i][j]), ff), q1 = mul2(bf16x2_to_f32x2(xr[i][j + 1]), ff);
-                    out[j / 2] = cvt_fp8x4<ELEM>(q0.x, q0.y, q1.x, q1.y);
-                }
-            } else {
-                const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
-#pragma unroll
-                for (int j = 0; j < W; j += 2) {
-                    const float2 q0 = mul2(mul2(bf16x2_to_f32x2(xr[i][j]), rr), ii);
-                    const float2 q1 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 1]), rr), ii);
-                    out[j / 2] = cvt_fp8x4<ELEM>(q0.x, q0.y, q1.x, q1.y);
-                }
-            }
+            sb = quantise_piece_fp8<B, PAPER, ELEM>(xr[i], m[i], rho, rho_normal, active, P.round, out);
         } else {
             // y = fl32(fl32(x*rho) * gamma); scales and codes from y
             uint32_t gr[W];
@@ -279,32 +360,8 @@ __device__ __forceinline__ void quantise_store_mxfp4(const uint32_t (&xr)[NPASS]
     for (int i = 0; i < NPASS; ++i) {
         const int k = (i * WPR + w) * kWarp + lane;
         const bool active = k < P.chunks;
-        const float a = __fmul_rn(m[i], rho);
-        const uint32_t u = __float_as_uint(a), E = u >> 23;
-        uint32_t sb;
-        if (E >= 255u) sb = (u & 0x7FFFFFu) ? 0u : 254u;   // not finite (outside the contract)
-        else sb = (uint32_t)max((int)E + ((u & 0x7FFFFFu) != 0u) - 2, 0);
-        const float inv = inv_scale(sb);
-        const float f = __fmul_rn(rho, inv);
-        const bool fast = sb >= 16u && rho_normal && is_normal_f32(f);   // same argument as for E4M3
         uint32_t out[W / 4];
-        if (__all_sync(0xFFFFFFFFu, fast || !active)) {
-            const float2 ff = make_float2(f, f);
-#pragma unroll
-            for (int j = 0; j < W; j += 4) {
-                const float2 q0 = mul2(bf16x2_to_f32x2(xr[i][j]), ff), q1 = mul2(bf16x2_to_f32x2(xr[i][j + 1]), ff);
-                const float2 q2 = mul2(bf16x2_to_f32x2(xr[i][j + 2]), ff), q3 = mul2(bf16x2_to_f32x2(xr[i][j + 3]), ff);
-                out[j / 4] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
-            }
-        } else {
-            const float2 rr = make_float2(rho, rho), ii = make_float2(inv, inv);
-#pragma unroll
-            for (int j = 0; j < W; j += 4) {
-                const float2 q0 = mul2(mul2(bf16x2_to_f32x2(xr[i][j]), rr), ii), q1 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 1]), rr), ii);
-                const float2 q2 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 2]), rr), ii), q3 = mul2(mul2(bf16x2_to_f32x2(xr[i][j + 3]), rr), ii);
-                out[j / 4] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
-            }
-        }
+        const uint32_t sb = quantise_piece_mxfp4<B>(xr[i], m[i], rho, rho_normal, active, out);
         if (active) {
             uint8_t* cp = cp0 + (int64_t)i * (WPR * kWarp * (B / 2));
             if (B == 16) st_v2(cp, out);
@@ -332,36 +389,96 @@ __device__ __forceinline__ void quantise_store_nvfp4(const uint32_t (&xr)[NPASS]
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
         const int k = (i * WPR + w) * kWarp + lane;
-        // block scale = E4M3(fl32(fl32(a/6) * global_scale)), a = fl32(m * rho~);
-        // element factor = fl32(rho~ * global_scale) / scale (0 when the scale is 0)
-        const float a = __fmul_rn(m[i], rho);
-        // the common case first, without the IEEE division sequences and decided for the whole warp at once:
-        // numerators inside the window of the exact shortcut and a normal E4M3 scale
-        uint32_t sc = cvt_e4m3x2(__fmul_rn(div_by_known(a, 6.0f, 0x1.555556p-3f), P.global_scale), 0.0f) & 0xFFu;
-        const bool common = in_division_window(a) && sc >= 8u && rho_g_in_window;
-        float inv;
-        if (__all_sync(0xFFFFFFFFu, common || k >= P.K)) {
-            const float d = __uint_as_float((sc << 20) + (120u << 23));            // (8+mf) * 2^(ef-10)
-            const float c = __fmul_rn(__shfl_sync(0xFFFFFFFFu, rcp_sig, (int)(sc & 7u)), __uint_as_float((134u - (sc >> 3)) << 23));
-            inv = div_by_known(rho_g, d, c);
-        } else {
-            sc = cvt_e4m3x2(__fmul_rn(div_by_6(a), P.global_scale), 0.0f) & 0xFFu;
-            const float d = e4m3_to_f32(sc);
-            if (sc >= 8u && rho_g_in_window) inv = div_by_e4m3_normal(rho_g, sc, d);
-            else inv = d == 0.0f ? 0.0f : fminf(__fdiv_rn(rho_g, d), 3.402823466e+38f);   // saturates like rho itself
-        }
         uint32_t out[2];
-        const float2 ii = make_float2(inv, inv);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t* xw = &xr[i][h * 4];
-            const float2 q0 = mul2(bf16x2_to_f32x2(xw[0]), ii), q1 = mul2(bf16x2_to_f32x2(xw[1]), ii);
-            const float2 q2 = mul2(bf16x2_to_f32x2(xw[2]), ii), q3 = mul2(bf16x2_to_f32x2(xw[3]), ii);
-            out[h] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
-        }
+        const uint32_t sc = quantise_piece_nvfp4(xr[i], m[i], rho, rho_g, rho_g_in_window, rcp_sig, P.global_scale, k < P.K, out);
         if (k < P.K) {
             st_v2(cp0 + (int64_t)i * (WPR * kWarp * 8), out);
             sp0[i * sstep] = (uint8_t)sc;
+        }
+    }
+}
+
+// NVFP4 with a lane owning two adjacent blocks (32 contiguous elements): the per-block scalar arithmetic of the two
+// blocks runs as packed binary32 pairs (each half an ordinary IEEE operation, so results are those of
+// quantise_piece_nvfp4 bit for bit), both E4M3 scale bytes come out of one conversion and leave as one 16-bit store,
+// and the 32 codes leave as one 16-byte store.  Every lane of the warp must call.
+__device__ __forceinline__ float2 div2_by_known(float2 a, float2 d, float2 c)
+{
+    const float2 q = __fmul2_rn(a, c);
+    const float2 r = __ffma2_rn(make_float2(-d.x, -d.y), q, a);
+    return __ffma2_rn(r, c, q);
+}
+__device__ __forceinline__ uint32_t quantise_pair_nvfp4(const uint32_t (&x)[16], float m0, float m1, float rho, float rho_g,
+                                                        bool rho_g_in_window, float rcp_sig, float global_scale, bool active,
+                                                        uint32_t (&out)[4])
+{
+    const float2 a = __fmul2_rn(make_float2(m0, m1), make_float2(rho, rho));
+    const float2 six = make_float2(6.0f, 6.0f), c6 = make_float2(0x1.555556p-3f, 0x1.555556p-3f), gs = make_float2(global_scale, global_scale);
+    const float2 t = __fmul2_rn(div2_by_known(a, six, c6), gs);
+    uint32_t sc2 = cvt_e4m3x2(t.x, t.y);                 // block 0 in the low byte
+    uint32_t sc0 = sc2 & 0xFFu, sc1 = sc2 >> 8;
+    const bool common = in_division_window(a.x) && in_division_window(a.y) && sc0 >= 8u && sc1 >= 8u && rho_g_in_window;
+    float2 inv;
+    if (__all_sync(0xFFFFFFFFu, common || !active)) {
+        const float2 d = make_float2(__uint_as_float((sc0 << 20) + (120u << 23)), __uint_as_float((sc1 << 20) + (120u << 23)));
+        const float2 c = make_float2(
+            __fmul_rn(__shfl_sync(0xFFFFFFFFu, rcp_sig, (int)(sc0 & 7u)), __uint_as_float((134u - (sc0 >> 3)) << 23)),
+            __fmul_rn(__shfl_sync(0xFFFFFFFFu, rcp_sig, (int)(sc1 & 7u)), __uint_as_float((134u - (sc1 >> 3)) << 23)));
+        inv = div2_by_known(make_float2(rho_g, rho_g), d, c);
+    } else {
+        float iv[2];
+        uint32_t sc[2];
+        const float av[2] = {a.x, a.y};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            sc[h] = cvt_e4m3x2(__fmul_rn(div_by_6(av[h]), global_scale), 0.0f) & 0xFFu;
+            const float d = e4m3_to_f32(sc[h]);
+            if (sc[h] >= 8u && rho_g_in_window) iv[h] = div_by_e4m3_normal(rho_g, sc[h], d);
+            else iv[h] = d == 0.0f ? 0.0f : fminf(__fdiv_rn(rho_g, d), 3.402823466e+38f);
+        }
+        sc0 = sc[0];
+        sc1 = sc[1];
+        sc2 = sc0 | (sc1 << 8);
+        inv = make_float2(iv[0], iv[1]);
+    }
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const float f = h < 2 ? inv.x : inv.y;
+        const float2 ii = make_float2(f, f);
+        const uint32_t* xw = &x[h * 4];
+        const float2 q0 = mul2(bf16x2_to_f32x2(xw[0]), ii), q1 = mul2(bf16x2_to_f32x2(xw[1]), ii);
+        const float2 q2 = mul2(bf16x2_to_f32x2(xw[2]), ii), q3 = mul2(bf16x2_to_f32x2(xw[3]), ii);
+        out[h] = cvt_e2m1x8(q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y);
+    }
+    return sc2;
+}
+
+// phase 2 of the pair kernel: lane `lane` of pass i of warp w owns blocks 2k and 2k+1, k = (i*WPR + w)*32 + lane
+template <int NPASS, int WPR>
+__device__ __forceinline__ void quantise_store_nvfp4_pair(const uint32_t (&xr)[NPASS][16], const float (&m0)[NPASS], const float (&m1)[NPASS],
+                                                          float rho, const FwdParams& P, int64_t row, int w, int lane)
+{
+    const float rho_g = __fmul_rn(rho, P.global_scale);
+    const bool rho_g_in_window = in_division_window(rho_g);
+    const float rcp_sig = kRcpE4M3Significand[lane & 7];
+    uint8_t* cp0 = P.codes + row * (P.D / 2) + (int64_t)(w * kWarp + lane) * 16;
+#pragma unroll
+    for (int i = 0; i < NPASS; ++i) {
+        const int k = (i * WPR + w) * kWarp + lane;
+        const bool active = k < P.chunks;
+        uint32_t out[4];
+        const uint32_t sc2 = quantise_pair_nvfp4(xr[i], m0[i], m1[i], rho, rho_g, rho_g_in_window, rcp_sig, P.global_scale, active, out);
+        if (active) {
+            st_v4(cp0 + (int64_t)i * (WPR * kWarp * 16), out);
+            const int kb = 2 * k;
+            int64_t off;
+            if (P.layout == MXN_SCALES_ROWMAJOR) {
+                off = row * P.K + kb;
+            } else {
+                const int rr = (int)(row & 127);
+                off = ((row >> 7) * P.tiles_per_row + (kb >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (kb & 3);
+            }
+            *reinterpret_cast<uint16_t*>(P.scales + off) = (uint16_t)sc2;      // two adjacent scale bytes (off is even)
         }
     }
 }
