@@ -37,10 +37,11 @@ WORKLOAD = "C3"
 EPS = 1e-5
 SETS = 4            # rotating input/output buffer sets: 4 x 203 MB > 126 MB of L2
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one mxnorm_fwd launch at [16384, 4096], from the
-# committed ncu summary profiles/mxnorm_fwd_c3_ncu_full.md (134.24 MB read + 35.94 MB written; the
-# rest of the 69.3 MB of output is still dirty in L2 when the kernel ends)
-NCU_TRAFFIC_BYTES = 170_177_280
+REPEATS = 5         # the timed region (K launches) is repeated this often; the median repeat is the headline
+# dram__bytes_read.sum + dram__bytes_write.sum per mxnorm_fwd launch at [16384, 4096]: the mean over eight consecutive
+# launches that rotate over the buffer sets, captured with ncu in steady state (caches not flushed between launches)
+NCU_TRAFFIC_BYTES = 202_970_368
+NCU_TRAFFIC_KIND = "ncu, mean of 8 consecutive launches rotating over the buffer sets (steady state)"
 
 
 def algorithmic_bytes(kind: str, T: int, D: int) -> int:
@@ -51,6 +52,12 @@ def algorithmic_bytes(kind: str, T: int, D: int) -> int:
     if kind == "bwd":
         return 3 * T * D * 2 + 4 * T + 2 * D + 4 * D
     raise ValueError(kind)
+
+
+def workload_name(T: int, D: int) -> str:
+    """The same string in both arms (the GPU path and the CPU oracle run the same workload)."""
+    return (f"{WORKLOAD}: mxnorm_fwd bf16 [{T},{D}] per GPU (batch 4 x seq 4096, Llama-3-8B hidden), outlier channels, "
+            "MXFP8 E4M3 codes + E8M0 scales (B=32) in the 128x4 tiled GEMM layout, p=2")
 
 
 def measured_peak():
@@ -124,6 +131,21 @@ def time_launches(fn, n_sets: int, steps: int, warmup: int, stream) -> float:
     end.record(stream)
     torch.cuda.synchronize()
     return start.elapsed_time(end) / steps
+
+
+def time_repeated(fn, n_sets: int, steps: int, warmup: int, stream, repeats: int = REPEATS):
+    """`repeats` timed regions of `steps` launches each (one warm-up phase); returns the per-launch milliseconds of every
+    repeat, sorted."""
+    out = [time_launches(fn, n_sets, steps, warmup if r == 0 else 0, stream) for r in range(repeats)]
+    return sorted(out)
+
+
+def time_median(fn, n_sets: int, steps: int, warmup: int, stream, repeats: int = 3) -> float:
+    return statistics.median(time_repeated(fn, n_sets, steps, warmup, stream, repeats))
+
+
+def spread(ms_sorted):
+    return {"median": statistics.median(ms_sorted), "min": ms_sorted[0], "max": ms_sorted[-1], "repeats": len(ms_sorted)}
 
 
 def time_graph_replay(fn, n_sets: int, steps: int, warmup: int, stream) -> float:
@@ -252,7 +274,7 @@ def run_reference(args, rank: int):
         "impl": "reference", "metric": "mxnorm_fwd_hbm_gbs_d4096", "value": gbs, "unit": "GB/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD} bf16 [{w.T},{w.D}] MXFP8 B=32, CPU oracle (plain C, fp64 statistics)"},
+        "config": {"workload": workload_name(w.T, w.D), "impl_note": "CPU oracle mxnorm_ref (plain C, binary64 statistics, OpenMP over rows)"},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
                          "sample": f"the full [{w.T},{w.D}] batch per step"},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -336,8 +358,9 @@ def main():
         time.sleep(0.3)
     if dist is not None:
         dist.barrier()
-    ms = time_launches(fwd, SETS, args.steps, args.warmup, stream)
-    ms = sharding.max_over_ranks(ms, device="cuda")
+    reps = time_repeated(fwd, SETS, args.steps, args.warmup, stream)      # REPEATS regions of exactly K launches each
+    reps = sorted(sharding.max_over_ranks(v, device="cuda") for v in reps)   # max over ranks, repeat by repeat
+    ms = statistics.median(reps)
     # keep the GPU under load a little longer so that the 50 ms sampler sees it
     if rank == 0:
         t_end = time.time() + 0.5
@@ -354,7 +377,7 @@ def main():
         marker.record(stream)
 
     marker = torch.cuda.Event()
-    ms_serial = time_launches(fwd_serialised, SETS, args.steps, args.warmup, stream)
+    ms_serial = time_median(fwd_serialised, SETS, args.steps, args.warmup, stream)
 
     nbytes = algorithmic_bytes("mx", T, D)
     gbs_one = nbytes / (ms * 1e-3) / 1e9
@@ -363,29 +386,32 @@ def main():
         "metric": "mxnorm_fwd_hbm_gbs_d4096", "value": gbs_one * world, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: mxnorm_fwd bf16 [{T},{D}] per GPU (batch 4 x seq 4096, Llama-3-8B hidden), "
-                               "outlier channels, MXFP8 E4M3 codes + E8M0 scales (B=32) in the 128x4 tiled GEMM layout, p=2",
+        "config": {"workload": workload_name(T, D),
                    "l2": f"inputs/outputs rotate over {SETS} buffer sets ({SETS * nbytes / 1e6:.0f} MB > 126 MB L2)",
+                   "timing": f"{REPEATS} timed regions of {args.steps} launches each after {args.warmup} warm-up launches; ms_per_step "
+                             "is the median region, ms_per_step_spread its minimum and maximum; the other kernels: median of 3 regions",
                    "launch": "back-to-back launches in one stream, as the library issues them: programmatic stream "
                              "serialisation (each kernel waits for the previous one before it reads or writes any value; launch "
                              "latency and L2 prefetch hints for the first-wave rows overlap the previous kernel's tail); "
                              "event_between_launches_ms_per_step records an event after every launch",
                    "parallelism": f"rows sharded, no collective (x{world})"},
+        "ms_per_step_spread": spread(reps),
         "event_between_launches_ms_per_step": ms_serial,
         "tokens_per_s": T * world / (ms * 1e-3),
         "gpu_launches": args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": gbs_one, "peak": peak, "unit": "GB/s", "frac": gbs_one / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_8TBs": gbs_one / 8000.0,
-                     "traffic": NCU_TRAFFIC_BYTES if T == w.T else None, "algorithmic_bytes": nbytes,
+                     "traffic": NCU_TRAFFIC_BYTES if T == w.T else None, "traffic_kind": NCU_TRAFFIC_KIND,
+                     "algorithmic_bytes": nbytes,
                      "kernel": "fwd_e4m3_kernel<B=32,NPASS=2,WPR=2,STAT=MX>"},
     }
 
     if not args.skip_others:
         # ---- the rest of the path, each timed the same way (context for the headline) ----
         others = {}
-        ms_rms = time_launches(rms, SETS, args.steps, args.warmup, stream)
-        ms_cast = time_launches(cast, SETS, args.steps, args.warmup, stream)
+        ms_rms = time_median(rms, SETS, args.steps, args.warmup, stream)
+        ms_cast = time_median(cast, SETS, args.steps, args.warmup, stream)
         others["rmsnorm_mxfp8_fwd"] = {"ms": ms_rms, "gbs": algorithmic_bytes("rms", T, D) / ms_rms / 1e6}
         others["mx_cast"] = {"ms": ms_cast, "gbs": algorithmic_bytes("cast", T, D) / ms_cast / 1e6}
         result["speedup_vs_rmsnorm_mxfp8_fwd"] = ms_rms / ms
@@ -405,8 +431,8 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            ms4 = time_launches(nvfp4, SETS, args.steps, args.warmup, stream)
-            ms4r = time_launches(rms_nvfp4, SETS, args.steps, args.warmup, stream)
+            ms4 = time_median(nvfp4, SETS, args.steps, args.warmup, stream)
+            ms4r = time_median(rms_nvfp4, SETS, args.steps, args.warmup, stream)
             others["mxnorm_nvfp4_fwd"] = {"ms": ms4, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4 / 1e6}
             others["rmsnorm_nvfp4_fwd"] = {"ms": ms4r, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4r / 1e6}
             result["nvfp4_speedup_vs_rmsnorm_nvfp4_fwd"] = ms4r / ms4
@@ -420,7 +446,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msm4 = time_launches(mxfp4, SETS, args.steps, args.warmup, stream)
+            msm4 = time_median(mxfp4, SETS, args.steps, args.warmup, stream)
             others["mxnorm_mxfp4_fwd"] = {"ms": msm4, "gbs": (T * D * 2 + T * D // 2 + T * (D // 32) + 4 * T) / msm4 / 1e6}
             del m4
             if T % 32 == 0:
@@ -433,7 +459,7 @@ def main():
                     if st != 0:
                         raise RuntimeError(mx.status_string(st))
 
-                mst = time_launches(transposed, SETS, args.steps, args.warmup, stream)
+                mst = time_median(transposed, SETS, args.steps, args.warmup, stream)
                 others["mx_cast_transposed"] = {"ms": mst, "gbs": (T * D * 3 + T * D // 32 + 4 * T) / mst / 1e6}
                 del ct, stt
             # the ablation with power-of-two-rounded block maxima, and the residual add fused in front
@@ -443,7 +469,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            mspr = time_launches(postround, SETS, args.steps, args.warmup, stream)
+            mspr = time_median(postround, SETS, args.steps, args.warmup, stream)
             others["mxnorm_postround_fwd"] = {"ms": mspr, "gbs": algorithmic_bytes("mx", T, D) / mspr / 1e6}
             hs = [torch.empty_like(xs[0]) for _ in range(SETS)]
 
@@ -454,7 +480,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msadd = time_launches(add_fwd, SETS, args.steps, args.warmup, stream)
+            msadd = time_median(add_fwd, SETS, args.steps, args.warmup, stream)
             others["mxnorm_add_fwd"] = {"ms": msadd, "gbs": (algorithmic_bytes("mx", T, D) + 4 * T * D) / msadd / 1e6}
             del hs
             # backward (C5 tensors: seed 1, gradient ~ N(0, 1e-2), gain)
@@ -477,7 +503,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msb = time_launches(bwd, nb, max(10, args.steps // 2), args.warmup, stream)
+            msb = time_median(bwd, nb, max(10, args.steps // 2), args.warmup, stream)
             others["mxnorm_bwd"] = {"ms": msb, "gbs": algorithmic_bytes("bwd", T, D) / msb / 1e6}
 
             def bwd_dx_only(i):   # the method's own configuration: no gain (folded into the next weight), hence no gain gradient
@@ -485,7 +511,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msbx = time_launches(bwd_dx_only, nb, max(10, args.steps // 2), args.warmup, stream)
+            msbx = time_median(bwd_dx_only, nb, max(10, args.steps // 2), args.warmup, stream)
             others["mxnorm_bwd_dx_only"] = {"ms": msbx, "gbs": (3 * T * D * 2 + 4 * T) / msbx / 1e6}
             del xb, gb, dxb
 
