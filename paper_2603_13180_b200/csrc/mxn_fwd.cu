@@ -257,33 +257,34 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_nvf
     quantise_store_nvfp4_pair<NPASS, WPR>(xr, m0, m1, rho, P, row, w, lane);
 }
 
-// ---- several short rows per warp ----------------------------------------------------------------------------------
-// One warp, no shared memory: a row spans RSPAN passes of the warp (piece k of a row goes to pass k / 32, lane k % 32) and
-// the warp takes NPASS / RSPAN consecutive rows.  Pieces may be smaller than a block (E = 16 elements, LPB lanes per
-// block), which lets rows of 5 * 2^r blocks fill whole passes of one warp.  The row statistics are independent shuffle
-// reductions, one per row.
-template <int E, int LPB, int NPASS, int RSPAN, int STAT, int FMT>
+// ---- one warp per run of RPW short rows ------------------------------------------------------------------------------
+// One warp, no shared memory.  The warp takes RPW consecutive rows of CH pieces each (E = 16 elements per piece, LPB lanes
+// per block) as one contiguous run of RPW * CH pieces: piece j of the run goes to pass j / 32, lane j % 32, so every lane
+// of every pass is busy when RPW * CH = 32 NPASS, however the rows fall on the passes (CH is a compile-time constant:
+// the row of a piece is a constant division).  Used for rows of 5 * 2^r blocks that no warps-per-row split fills:
+// D = 2560 (CH = 160, one row per warp) and D = 1280 (CH = 80, two rows per warp).  The row statistics are independent
+// shuffle reductions, one per row.
+template <int E, int LPB, int NPASS, int RPW, int CH, int STAT, int FMT>
 __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_multi_kernel(const FwdParams P)
 {
-    constexpr int W = E / 2, RPW = NPASS / RSPAN;
-    static_assert(NPASS % RSPAN == 0 && (E == 16 || E == 32), "whole rows per warp; 32- or 64-byte pieces");
+    constexpr int W = E / 2;
+    static_assert(RPW * CH <= 32 * NPASS && CH % LPB == 0 && (E == 16 || E == 32), "the run fits the warp's passes; 32- or 64-byte pieces");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row0 = ((int64_t)blockIdx.x * MXN_FWD_WARPS + warp) * RPW;
-    if (lane == 0 && blockIdx.x < kFirstWaveCtas && row0 < P.T) {
-        const int64_t nrows = P.T - row0 < RPW ? P.T - row0 : RPW;
-        prefetch_l2_bulk(P.x + row0 * P.D, (uint32_t)(nrows * P.D) * 2u);
-    }
+    const int nrows = (int)(P.T - row0 < RPW ? P.T - row0 : RPW);     // <= 0 past the end
+    if (lane == 0 && blockIdx.x < kFirstWaveCtas && nrows > 0) prefetch_l2_bulk(P.x + row0 * P.D, (uint32_t)(nrows * CH) * (E * 2u));
     pdl_prologue();
-    if (row0 >= P.T) return;
+    if (nrows <= 0) return;
+    const int npieces = nrows * CH;
+    const int64_t first = row0 * CH;
 
     uint32_t xr[NPASS][W];
     float m[NPASS];
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
-        const int64_t row = row0 + i / RSPAN;
-        const int k = (i % RSPAN) * 32 + lane;
-        if (row < P.T && k < P.chunks) {
-            const uint16_t* p = P.x + row * P.D + (int64_t)k * E;
+        const int j = i * 32 + lane;
+        if (j < npieces) {
+            const uint16_t* p = P.x + (first + j) * E;
 #pragma unroll
             for (int v = 0; v < W / 8; ++v) ld_v8(p + v * 16, &xr[i][v * 8]);
         } else {
@@ -292,13 +293,15 @@ __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_mult
         }
     }
     double stat[RPW];
-#pragma unroll
-    for (int r = 0; r < RPW; ++r) stat[r] = 0.0;
     float2 ssa[RPW], ssb[RPW];
 #pragma unroll
-    for (int r = 0; r < RPW; ++r) ssa[r] = ssb[r] = make_float2(0.f, 0.f);
+    for (int r = 0; r < RPW; ++r) {
+        stat[r] = 0.0;
+        ssa[r] = ssb[r] = make_float2(0.f, 0.f);
+    }
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
+        const int rl = (i * 32 + lane) / CH;
         uint32_t m2 = absmax_bf16x2(xr[i][0], xr[i][1]);
 #pragma unroll
         for (int q = 2; q < W; ++q) m2 = absmax_bf16x2(m2, xr[i][q]);
@@ -306,16 +309,26 @@ __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_mult
 #pragma unroll
         for (int o = 1; o < LPB; o <<= 1) m[i] = fmaxf(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], o));
         const float mc = (LPB == 1 || (lane & (LPB - 1)) == 0) ? m[i] : 0.0f;
-        if (STAT == STAT_MX) {
-            const double md = (double)mc;
-            stat[i / RSPAN] = P.p == 2 ? __fma_rn(md, md, stat[i / RSPAN]) : __dadd_rn(stat[i / RSPAN], md);
-        }
+        float2 sa = make_float2(0.f, 0.f), sb2 = make_float2(0.f, 0.f);
         if (STAT == STAT_RMS) {
 #pragma unroll
             for (int q = 0; q < W; q += 2) {
                 const float2 a = bf16x2_to_f32x2(xr[i][q]), b = bf16x2_to_f32x2(xr[i][q + 1]);
-                ssa[i / RSPAN] = __ffma2_rn(a, a, ssa[i / RSPAN]);
-                ssb[i / RSPAN] = __ffma2_rn(b, b, ssb[i / RSPAN]);
+                sa = __ffma2_rn(a, a, sa);
+                sb2 = __ffma2_rn(b, b, sb2);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            if (i * 32 / CH > r || (i * 32 + 31) / CH < r) continue;       // this pass holds no piece of row r (compile time)
+            const bool mine = RPW == 1 || rl == r;
+            if (STAT == STAT_MX) {
+                const double md = mine ? (double)mc : 0.0;                    // adding 0 is exact
+                stat[r] = P.p == 2 ? __fma_rn(md, md, stat[r]) : __dadd_rn(stat[r], md);
+            }
+            if (STAT == STAT_RMS) {
+                ssa[r] = __fadd2_rn(ssa[r], mine ? sa : make_float2(0.f, 0.f));
+                ssb[r] = __fadd2_rn(ssb[r], mine ? sb2 : make_float2(0.f, 0.f));
             }
         }
     }
@@ -328,22 +341,24 @@ __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_mult
             if (STAT == STAT_RMS) stat[r] = (double)ssa[r].x + (double)ssa[r].y + ((double)ssb[r].x + (double)ssb[r].y);
             float rr;
             finish_stat<STAT>(warp_sum(stat[r]), P, rr, rho[r]);
-            if (P.rms_out != nullptr && lane == 0 && row0 + r < P.T) P.rms_out[row0 + r] = rr;
+            if (P.rms_out != nullptr && lane == 0 && r < nrows) P.rms_out[row0 + r] = rr;
         }
     }
     const float rcp_sig = FMT == 2 ? kRcpE4M3Significand[lane & 7] : 0.0f;
 #pragma unroll
     for (int i = 0; i < NPASS; ++i) {
-        const int64_t row = row0 + i / RSPAN;
-        const int k = (i % RSPAN) * 32 + lane;
-        const bool active = row < P.T && k < P.chunks;
-        const float rh = rho[i / RSPAN];
+        const int j = i * 32 + lane;
+        const bool active = j < npieces;
+        const int rl = j / CH;
+        float rh = rho[0];
+#pragma unroll
+        for (int r = 1; r < RPW; ++r) rh = rl == r ? rho[r] : rh;
         uint32_t sbyte;
         if constexpr (FMT == 0) {
             uint32_t out[W / 2];
             sbyte = quantise_piece_fp8<E, true, 0>(xr[i], m[i], rh, is_normal_f32(rh), active, 0, out);
             if (active) {
-                uint8_t* cp = P.codes + row * P.D + (int64_t)k * E;
+                uint8_t* cp = P.codes + (first + j) * E;
                 if constexpr (E == 16) st_v4(cp, out);
                 else st_v8(cp, out);
             }
@@ -351,7 +366,7 @@ __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_mult
             uint32_t out[W / 4];
             sbyte = quantise_piece_mxfp4<E>(xr[i], m[i], rh, is_normal_f32(rh), active, out);
             if (active) {
-                uint8_t* cp = P.codes + row * (P.D / 2) + (int64_t)k * (E / 2);
+                uint8_t* cp = P.codes + (first + j) * (E / 2);
                 if constexpr (E == 16) st_v2(cp, out);
                 else st_v4(cp, out);
             }
@@ -359,15 +374,15 @@ __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_mult
             uint32_t out[2];
             const float rho_g = __fmul_rn(rh, P.global_scale);
             sbyte = quantise_piece_nvfp4(xr[i], m[i], rh, rho_g, in_division_window(rho_g), rcp_sig, P.global_scale, active, out);
-            if (active) st_v2(P.codes + row * (P.D / 2) + (int64_t)k * 8, out);
+            if (active) st_v2(P.codes + (first + j) * 8, out);
         }
         if (active && (LPB == 1 || (lane & (LPB - 1)) == 0)) {
-            const int kb = k / LPB;
             int64_t off;
             if (P.layout == MXN_SCALES_ROWMAJOR) {
-                off = row * P.K + kb;
+                off = (first + j) / LPB;                       // scales of consecutive rows are contiguous too
             } else {
-                const int rr = (int)(row & 127);
+                const int64_t row = row0 + rl;
+                const int kb = (j - rl * CH) / LPB, rr = (int)(row & 127);
                 off = ((row >> 7) * P.tiles_per_row + (kb >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (kb & 3);
             }
             P.scales[off] = (uint8_t)sbyte;
@@ -530,22 +545,30 @@ static fwd_fn pick_nvfp4(int wpr, int npass)
 }
 
 // The one-warp kernel with 16-element pieces is used where it measured faster than the row-group kernels: rows of
-// exactly 160 pieces (D = 2560), five passes of one warp instead of three warps x one pass or two warps x four passes
-// ([16384, 2560]: 5.7 -> 5.9 TB/s for blocks of 32, 5.3 -> 6.1 for blocks of 16, NVFP4 4.5 -> 5.1).  Measured and not
-// kept: two rows of 32 pieces per warp (D = 1024: 5.5 -> 5.2 TB/s), three passes of 16-element pieces (D = 1536:
-// 5.8 -> 5.5) and 8-element pieces, four lanes per block (D = 1280: 5.1 -> 3.8, D = 1792: 6.1 -> 4.0).
-static bool use_one_warp_kernel(int64_t D, int B) { return D == 2560 && (B == 16 || B == 32 || B == 64); }
+// 160 pieces (D = 2560: five passes of one warp instead of three warps x one pass or two warps x four passes;
+// [16384, 2560]: 5.7 -> 5.9 TB/s for blocks of 32, 5.3 -> 6.1 for blocks of 16, NVFP4 4.5 -> 5.1) and rows of 80 pieces
+// (D = 1280: two rows per warp; NVFP4 only: 4.2 -> 4.5 TB/s at 16384 rows, 4.9 -> 5.5 at 65536, while the E8M0-scaled
+// formats lose 1-5 % there).  Measured and not kept: two rows of 32 pieces per warp (D = 1024: 5.5 -> 5.2 TB/s),
+// three passes of 16-element pieces (D = 1536: 5.8 -> 5.5), 8-element pieces with four lanes per block (D = 1280:
+// 5.1 -> 3.8, D = 1792: 6.1 -> 4.0), and CTA tiles of whole rows packed across warps through shared memory (two
+// CTA-wide barriers per tile: slower than one row per row group at every size but D = 2560).
+static int one_warp_rows(int64_t D, bool nvfp4) { return D == 2560 ? 1 : (D == 1280 && nvfp4) ? 2 : 0; }
 
-template <int FMT, int STAT>
-static fwd_fn pick_multi(int B)
+template <int LPB, int FMT, int STAT>
+static fwd_fn multi_by_rows(int rpw)
 {
-    if constexpr (FMT == 2) return fwd_multi_kernel<16, 1, 5, 5, STAT, 2>;
-    else return B == 16 ? fwd_multi_kernel<16, 1, 5, 5, STAT, FMT> : B == 32 ? fwd_multi_kernel<16, 2, 5, 5, STAT, FMT> : fwd_multi_kernel<16, 4, 5, 5, STAT, FMT>;
+    return rpw == 1 ? fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT> : fwd_multi_kernel<16, LPB, 5, 2, 80, STAT, FMT>;
+}
+template <int FMT, int STAT>
+static fwd_fn pick_multi(int B, int rpw)
+{
+    if constexpr (FMT == 2) return multi_by_rows<1, 2, STAT>(rpw);
+    else return B == 16 ? multi_by_rows<1, FMT, STAT>(rpw) : B == 32 ? multi_by_rows<2, FMT, STAT>(rpw) : multi_by_rows<4, FMT, STAT>(rpw);
 }
 template <int FMT>
-static fwd_fn pick_multi_stat(int B, int stat)
+static fwd_fn pick_multi_stat(int B, int stat, int rpw)
 {
-    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B) : pick_multi<FMT, STAT_NONE>(B);
+    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B, rpw) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B, rpw) : pick_multi<FMT, STAT_NONE>(B, rpw);
 }
 
 template <int NPASS, int STAT>
@@ -640,12 +663,10 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     P.rows_per_cta = rows_per_cta(P.wpr);
     const bool has_gain = P.gain != nullptr;
     fwd_fn fn = nullptr;
-    if ((fine || mxfp4) && stat != STAT_POSTROUND && use_one_warp_kernel(P.D, B)) {
-        constexpr int kE = 16, kPasses = 5;
-        fn = nvfp4 ? pick_multi_stat<2>(16, stat) : mxfp4 ? pick_multi_stat<1>(B, stat) : pick_multi_stat<0>(B, stat);
-        P.chunks = (int)(P.D / kE);
-        (void)kPasses;
-        const int64_t ctas = (P.T + MXN_FWD_WARPS - 1) / MXN_FWD_WARPS;
+    if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && (fine || mxfp4) && stat != STAT_POSTROUND) {
+        fn = nvfp4 ? pick_multi_stat<2>(16, stat, rpw) : mxfp4 ? pick_multi_stat<1>(B, stat, rpw) : pick_multi_stat<0>(B, stat, rpw);
+        const int64_t rows_per_cta = (int64_t)MXN_FWD_WARPS * rpw;
+        const int64_t ctas = (P.T + rows_per_cta - 1) / rows_per_cta;
         if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)ctas);

@@ -6,13 +6,19 @@ torch.compile kernels on a GB200).
 
 Each case is timed as the replay of a CUDA graph of back-to-back launches over rotating buffer sets (3x L2).
 
-    python -m paper_2603_13180_b200.sweep [--blocks 32] [--elem e4m3|e2m1|nvfp4] [--tokens 4096 16384 65536] [--json out.json]
+    python -m paper_2603_13180_b200.sweep [--blocks 32] [--elem e4m3|e2m1|nvfp4] [--tokens 4096 16384 65536] [--json out.json] [--md out.md]
+
+`--md` appends compact tables (one row per token count, one column per hidden size) to a Markdown file: bandwidth of
+`mxnorm_fwd` as a fraction of the measured copy peak, its speed-up over the conventional kernel, and - as a yardstick
+for the small cases, where a launch is too short to reach the peak whatever it does - the bandwidth of a plain
+device-to-device copy that moves the same number of bytes, timed the same way.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import math
+import os
 
 import torch
 
@@ -109,9 +115,19 @@ def _run(stream, tokens, hidden, blocks, steps, warmup, l2_bytes, elem, graph):
 
                 t_mx = min(_time(mxn, sets, steps, warmup, stream, graph) for _ in range(2))
                 t_rms = min(_time(rms, sets, steps, warmup, stream, graph) for _ in range(2))
+                # yardstick: a device-to-device copy of per_set / 2 bytes (it reads and writes them: per_set bytes of traffic)
+                half = per_set // 2 // 16 * 16
+                src = [torch.empty(half, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+                dst = [torch.empty(half, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+
+                def cpy(i):
+                    dst[i].copy_(src[i])
+
+                t_cp = min(_time(cpy, sets, steps, warmup, stream, graph) for _ in range(2))
                 rows.append({"elem": elem, "block": B, "tokens": T, "hidden": D, "mxnorm_us": t_mx, "rmsnorm_us": t_rms,
-                             "speedup": t_rms / t_mx, "mxnorm_gbs": per_set / t_mx / 1e3, "rmsnorm_gbs": per_set / t_rms / 1e3})
-                del xs, outs
+                             "speedup": t_rms / t_mx, "mxnorm_gbs": per_set / t_mx / 1e3, "rmsnorm_gbs": per_set / t_rms / 1e3,
+                             "copy_us": t_cp, "copy_gbs": 2 * half / t_cp / 1e3})
+                del xs, outs, src, dst
     return rows
 
 
@@ -130,6 +146,46 @@ def summarise(rows):
     return out
 
 
+def measured_peak_gbs() -> float:
+    """The machine's measured copy bandwidth (generated file at the repository root), else the stated fallback."""
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
+def markdown_tables(rows, peak: float) -> str:
+    """Compact tables per (element format, block size): rows = tokens, columns = hidden sizes."""
+    out = []
+    for elem in sorted({r["elem"] for r in rows}):
+        for B in sorted({r["block"] for r in rows if r["elem"] == elem}):
+            sel = [r for r in rows if r["elem"] == elem and r["block"] == B]
+            hidden = sorted({r["hidden"] for r in sel})
+            tokens = sorted({r["tokens"] for r in sel})
+            cell = {(r["tokens"], r["hidden"]): r for r in sel}
+            big = [r for r in sel if r["tokens"] >= 16384]
+            gm = math.exp(sum(math.log(r["speedup"]) for r in sel) / len(sel))
+            out.append(f"### {elem}, block {B}: {len(sel)} cases, geometric-mean speed-up {gm:.3f} "
+                       f"(max {max(r['speedup'] for r in sel):.3f}, min {min(r['speedup'] for r in sel):.3f})\n")
+            if big:
+                worst = min(big, key=lambda r: r["mxnorm_gbs"])
+                out.append(f"Lowest `mxnorm` bandwidth at 16384 tokens and more: {worst['mxnorm_gbs']:.0f} GB/s = {worst['mxnorm_gbs'] / peak:.2f} of the "
+                           f"measured peak at T = {worst['tokens']}, D = {worst['hidden']} (a copy of the same bytes: {worst['copy_gbs']:.0f} GB/s).\n")
+            for title, fn in (("`mxnorm` bandwidth / measured copy peak", lambda r: f"{r['mxnorm_gbs'] / peak:.2f}"),
+                              ("`mxnorm` microseconds per launch", lambda r: f"{r['mxnorm_us']:.1f}"),
+                              ("speed-up over the conventional kernel", lambda r: f"{r['speedup']:.2f}"),
+                              ("`mxnorm` bandwidth / bandwidth of a copy of the same bytes", lambda r: f"{r['mxnorm_gbs'] / r['copy_gbs']:.2f}")):
+                out.append(f"{title}:\n")
+                out.append("| tokens \\ hidden | " + " | ".join(str(h) for h in hidden) + " |")
+                out.append("|---|" + "---|" * len(hidden))
+                for T in tokens:
+                    out.append(f"| {T} | " + " | ".join(fn(cell[(T, h)]) if (T, h) in cell else "" for h in hidden) + " |")
+                out.append("")
+    return "\n".join(out) + "\n"
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--blocks", type=int, nargs="+", default=[32])
@@ -140,6 +196,7 @@ def main():
                     help="element format: e4m3/e2m1 with E8M0 scales, or nvfp4 (E2M1 codes, E4M3 scales, block 16)")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a CUDA-graph replay")
     ap.add_argument("--json", default="")
+    ap.add_argument("--md", default="", help="append compact Markdown tables to this file")
     args = ap.parse_args()
     rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps, elem=args.elem, graph=not args.no_graph)
     summary = summarise(rows)
@@ -150,6 +207,9 @@ def main():
     if args.json:
         with open(args.json, "w") as f:
             json.dump({"rows": rows, "summary": summary}, f)
+    if args.md:
+        with open(args.md, "a") as f:
+            f.write(markdown_tables(rows, measured_peak_gbs()))
 
 
 if __name__ == "__main__":
