@@ -460,15 +460,34 @@ static fwd_fn pick_round(int round, int stat, bool gain, int wpr, int npass)
 {
     return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, LPB, true>(stat, gain, wpr, npass) : pick_stat<B, LPB, false>(stat, gain, wpr, npass);
 }
+template <int B, int LPB, int NPASS, int STAT>
+static fwd_fn mxfp4_by_wpr(int wpr)
+{
+    switch (wpr) {
+        case 1: return fwd_mxfp4_kernel<B, NPASS, 1, STAT, LPB>;
+        case 2: return fwd_mxfp4_kernel<B, NPASS, 2, STAT, LPB>;
+        case 3: return fwd_mxfp4_kernel<B, NPASS, 3, STAT, LPB>;
+        case 4: return fwd_mxfp4_kernel<B, NPASS, 4, STAT, LPB>;
+        case 5: return fwd_mxfp4_kernel<B, NPASS, 5, STAT, LPB>;
+        case 6: return fwd_mxfp4_kernel<B, NPASS, 6, STAT, LPB>;
+        case 7: return fwd_mxfp4_kernel<B, NPASS, 7, STAT, LPB>;
+        case 8: return fwd_mxfp4_kernel<B, NPASS, 8, STAT, LPB>;
+        case 16: return fwd_mxfp4_kernel<B, NPASS, 16, STAT, LPB>;
+        default: return nullptr;
+    }
+}
+// the same set of (warps per row, passes) as the E4M3 headline kernels: every count in kFineWpr with the full pass
+// count, half of it (four-pass kernels) or one pass; one warp per row with any pass count
 template <int B, int LPB, int STAT>
 static fwd_fn pick_mxfp4(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr == 2) return fwd_mxfp4_kernel<B, MAXP, 2, STAT, LPB>;
-    if (wpr == 4) return fwd_mxfp4_kernel<B, MAXP, 4, STAT, LPB>;
-    if (wpr == 8) return fwd_mxfp4_kernel<B, MAXP, 8, STAT, LPB>;
-    if (wpr == 16) return fwd_mxfp4_kernel<B, MAXP, 16, STAT, LPB>;
-    if (wpr != 1) return nullptr;
+    if (wpr > 1) {
+        if (npass == MAXP) return mxfp4_by_wpr<B, LPB, MAXP, STAT>(wpr);
+        if (MAXP >= 4 && npass == MAXP / 2) return mxfp4_by_wpr<B, LPB, (MAXP >= 4 ? MAXP / 2 : 1), STAT>(wpr);
+        if (npass == 1) return mxfp4_by_wpr<B, LPB, 1, STAT>(wpr);
+        return nullptr;
+    }
     switch (npass) {
         case 1: return fwd_mxfp4_kernel<B, 1, 1, STAT, LPB>;
         case 2: return fwd_mxfp4_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, LPB>;
@@ -557,7 +576,8 @@ static int one_warp_rows(int64_t D, bool nvfp4) { return D == 2560 ? 1 : (D == 1
 template <int LPB, int FMT, int STAT>
 static fwd_fn multi_by_rows(int rpw)
 {
-    return rpw == 1 ? fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT> : fwd_multi_kernel<16, LPB, 5, 2, 80, STAT, FMT>;
+    if constexpr (FMT == 2) return rpw == 1 ? fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT> : fwd_multi_kernel<16, LPB, 5, 2, 80, STAT, FMT>;
+    else return rpw == 1 ? fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT> : nullptr;   // two rows per warp: NVFP4 only
 }
 template <int FMT, int STAT>
 static fwd_fn pick_multi(int B, int rpw)
@@ -649,7 +669,7 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     const bool nv_pair = nvfp4 && P.K % 2 == 0 && P.D < 12288;
 #endif
     const int E = nv_pair ? 32 : B == 64 ? 32 : B;   // elements per lane and pass; a block of 64 is shared by two lanes
-    const bool fine = nvfp4 || (!mxfp4 && !e5m2 && !add && stat != STAT_POSTROUND && P.gain == nullptr &&
+    const bool fine = nvfp4 || mxfp4 || (!e5m2 && !add && stat != STAT_POSTROUND && P.gain == nullptr &&
                                 P.round == MXN_ROUND_RCEIL_POW2);
     P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
     P.chunks = nv_pair ? P.K / 2 : P.K * (B / E);

@@ -115,13 +115,14 @@ def _run(stream, tokens, hidden, blocks, steps, warmup, l2_bytes, elem, graph):
 
                 t_mx = min(_time(mxn, sets, steps, warmup, stream, graph) for _ in range(2))
                 t_rms = min(_time(rms, sets, steps, warmup, stream, graph) for _ in range(2))
-                # yardstick: a device-to-device copy of per_set / 2 bytes (it reads and writes them: per_set bytes of traffic)
+                # yardstick: an elementwise copy kernel over per_set / 2 bytes (it reads and writes them: per_set bytes of
+                # traffic), as 32-bit words so that it is a plain vectorised kernel and not a copy-engine transfer
                 half = per_set // 2 // 16 * 16
-                src = [torch.empty(half, dtype=torch.uint8, device="cuda") for _ in range(sets)]
-                dst = [torch.empty(half, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+                src = [torch.zeros(half // 4, dtype=torch.int32, device="cuda") for _ in range(sets)]
+                dst = [torch.empty(half // 4, dtype=torch.int32, device="cuda") for _ in range(sets)]
 
                 def cpy(i):
-                    dst[i].copy_(src[i])
+                    torch.add(src[i], 1, out=dst[i])
 
                 t_cp = min(_time(cpy, sets, steps, warmup, stream, graph) for _ in range(2))
                 rows.append({"elem": elem, "block": B, "tokens": T, "hidden": D, "mxnorm_us": t_mx, "rmsnorm_us": t_rms,

@@ -67,15 +67,21 @@ def test_backward_config_full_size(binding, oracle):
     inp = wl.make_inputs(w)
     x, g, gain = wl.bits(inp["x"]), wl.bits(inp["grad"]), wl.bits(inp["gain"])
     _, _, rms = oracle.mxnorm_ref(x, eps=EPS)
-    # dgamma over all 16384 rows; dX on sampled rows (the oracle's column sum is a serial loop)
+    # dgamma over all 16384 rows (the oracle's column sum is a serial loop) and every row of dX (rows in parallel),
+    # compared chunk by chunk to bound the host memory of the binary64 reference
     dx, _, dg = run_bwd(binding, x, g, gain, rms, fp32_out=True)
     _, want_dg = oracle.mxnorm_bwd_ref(x, g, gain, rms, want_dx=False)
     assert np.all(np.abs(dg - want_dg) <= 1e-3 * np.abs(want_dg).max())
-    sel = np.unique(np.concatenate([np.arange(0, 16384, 257), [16383]]))
-    want_dx, _ = oracle.mxnorm_bwd_ref(x[sel], g[sel], gain, rms[sel], want_dgain=False)
-    scale = np.abs(want_dx).max(-1, keepdims=True)
-    assert np.all(np.abs(dx[sel] - want_dx) <= 1e-3 * scale)
     dxb, _, dg2 = run_bwd(binding, x, g, gain, rms, fp32_out=False)
-    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want_dx), 2.0 ** -126))) - 7)
-    assert np.all(np.abs(dxb[sel] - want_dx) <= ulp + 1e-3 * 2.0 ** -8 * scale)
     assert np.array_equal(dg, dg2)
+    worst = 0.0
+    for r0 in range(0, w.T, 2048):
+        sel = slice(r0, r0 + 2048)
+        want_dx, _ = oracle.mxnorm_bwd_ref(x[sel], g[sel], gain, rms[sel], want_dgain=False)
+        scale = np.abs(want_dx).max(-1, keepdims=True)
+        err = np.abs(dx[sel] - want_dx)
+        assert np.all(err <= 1e-3 * scale)
+        worst = max(worst, float((err / scale).max()))
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want_dx), 2.0 ** -126))) - 7)
+        assert np.all(np.abs(dxb[sel] - want_dx) <= ulp + 1e-3 * 2.0 ** -8 * scale)
+    assert worst < 1e-5          # in practice ~2e-7 of the row maximum

@@ -255,7 +255,8 @@ def test_rms_output_is_optional_and_stream_is_honoured(binding, oracle):
 
 
 @pytest.mark.parametrize("block", [16, 32, 64])
-@pytest.mark.parametrize("T,D", [(1, 64), (37, 768), (130, 1024), (33, 4096), (9, 2560), (5, 8192), (3, 16384), (257, 2048), (133, 1280)])
+@pytest.mark.parametrize("T,D", [(1, 64), (37, 768), (130, 1024), (33, 4096), (9, 2560), (5, 8192), (3, 16384), (257, 2048), (133, 1280),
+                                 (7, 3072), (6, 5120), (5, 6144), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (10, 1536), (6, 3584)])
 def test_mxfp4_matches_oracle(binding, oracle, T, D, block):
     """E2M1 codes with E8M0 scales (the paper's cast with the element type set to E2M1)."""
     x, _ = rows(T, D, seed=13 * T + D + block)
