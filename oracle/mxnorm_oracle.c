@@ -15,7 +15,7 @@
  * fused behind the text's back.
  *
  * Readings taken where the paper is silent or inconsistent are marked
- * [reading]; the project's design document lists them all.
+ * [reading] where they are taken.
  *
  * Pin status (see tests/test_oracle_pins.py): every function and branch below is pinned by something other
  * than itself - the paper's printed constants and bounds, closed forms, invariants, brute-force definitional

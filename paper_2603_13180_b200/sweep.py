@@ -22,7 +22,6 @@ import os
 
 import torch
 
-from . import binding as mx
 
 TOKENS = [2 ** 12, 2 ** 13, 2 ** 14, 2 ** 15, 2 ** 16]
 HIDDEN = sorted({k * 2 ** r for k in (1, 3, 5, 7) for r in range(4, 15) if 2 ** 10 <= k * 2 ** r <= 2 ** 14})
@@ -65,6 +64,7 @@ def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4
 
 
 def _run(stream, tokens, hidden, blocks, steps, warmup, l2_bytes, elem, graph):
+    from . import binding as mx   # needs the compiled library and a GPU; the table formatting below does not
     sh = stream.cuda_stream
     L = mx.lib
     rows = []
@@ -157,8 +157,9 @@ def measured_peak_gbs() -> float:
         return 6650.0
 
 
-def markdown_tables(rows, peak: float) -> str:
-    """Compact tables per (element format, block size): rows = tokens, columns = hidden sizes."""
+def markdown_tables(rows, peak: float, compact: bool = False) -> str:
+    """Compact tables per (element format, block size): rows = tokens, columns = hidden sizes
+    (compact: only the two bandwidth-fraction tables)."""
     out = []
     for elem in sorted({r["elem"] for r in rows}):
         for B in sorted({r["block"] for r in rows if r["elem"] == elem}):
@@ -178,6 +179,8 @@ def markdown_tables(rows, peak: float) -> str:
                               ("`mxnorm` microseconds per launch", lambda r: f"{r['mxnorm_us']:.1f}"),
                               ("speed-up over the conventional kernel", lambda r: f"{r['speedup']:.2f}"),
                               ("`mxnorm` bandwidth / bandwidth of a copy of the same bytes", lambda r: f"{r['mxnorm_gbs'] / r['copy_gbs']:.2f}")):
+                if compact and ("microseconds" in title or "speed-up" in title):
+                    continue
                 out.append(f"{title}:\n")
                 out.append("| tokens \\ hidden | " + " | ".join(str(h) for h in hidden) + " |")
                 out.append("|---|" + "---|" * len(hidden))
@@ -198,7 +201,17 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a CUDA-graph replay")
     ap.add_argument("--json", default="")
     ap.add_argument("--md", default="", help="append compact Markdown tables to this file")
+    ap.add_argument("--compact", action="store_true", help="with --md: only the two bandwidth-fraction tables per format")
+    ap.add_argument("--from-json", nargs="+", default=[], help="render --md from result files written by --json (no GPU needed)")
     args = ap.parse_args()
+    if args.from_json:
+        rows = []
+        for path in args.from_json:
+            with open(path) as f:
+                rows += json.load(f)["rows"]
+        with open(args.md, "a") as f:
+            f.write(markdown_tables(rows, measured_peak_gbs(), args.compact))
+        return
     rows = run(args.tokens, args.hidden, args.blocks, steps=args.steps, elem=args.elem, graph=not args.no_graph)
     summary = summarise(rows)
     for r in rows:
@@ -210,7 +223,7 @@ def main():
             json.dump({"rows": rows, "summary": summary}, f)
     if args.md:
         with open(args.md, "a") as f:
-            f.write(markdown_tables(rows, measured_peak_gbs()))
+            f.write(markdown_tables(rows, measured_peak_gbs(), args.compact))
 
 
 if __name__ == "__main__":
