@@ -461,6 +461,14 @@ def main():
 
                 mst = time_median(transposed, SETS, args.steps, args.warmup, stream)
                 others["mx_cast_transposed"] = {"ms": mst, "gbs": (T * D * 3 + T * D // 32 + 4 * T) / mst / 1e6}
+
+                def transposed_plain(i):   # no normaliser: the column-wise cast of the upstream gradient
+                    st = L.mx_cast_transposed(xs[i].data_ptr(), None, T, D, 0.0, ct[i].data_ptr(), stt[i].data_ptr(), 0, layout, sh)
+                    if st != 0:
+                        raise RuntimeError(mx.status_string(st))
+
+                mstp = time_median(transposed_plain, SETS, args.steps, args.warmup, stream)
+                others["mx_cast_transposed_no_normaliser"] = {"ms": mstp, "gbs": (T * D * 3 + T * D // 32) / mstp / 1e6}
                 del ct, stt
             # the ablation with power-of-two-rounded block maxima, and the residual add fused in front
             def postround(i):

@@ -10,10 +10,30 @@ namespace mxn {
 // xr[r] = the bf16 pair (column c, column c+1) of token r of the block; rho = 32 per-token factors in shared
 // memory (16-byte aligned).  y = fl32(x * rho_r); one E8M0 scale per column from max_r |y|; codes of
 // fl32(y * 2^(127-sb)).  out0/out1 = the 32 code bytes of column c / c+1 in token order.
-template <bool PAPER, int ELEM>
+// RHO = false: no per-token factor (rho = 1, e.g. the upstream gradient): the column maxima come from packed bf16
+// comparisons and every code from one product - the same results as RHO = true with factors of 1, at half the work.
+template <bool PAPER, int ELEM, bool RHO = true>
 __device__ __forceinline__ void quantise_column_pair(const uint32_t (&xr)[32], const float* rho, int round,
                                                      uint32_t (&out0)[8], uint32_t (&out1)[8], uint32_t& sb0, uint32_t& sb1)
 {
+    if constexpr (!RHO) {
+        uint32_t m2 = xr[0] & 0x7FFF7FFFu;
+#pragma unroll
+        for (int r = 1; r < 32; ++r) m2 = absmax_bf16x2(m2, xr[r]);     // per half: max(|a|, |b|); the sign bit is not used
+        const float m0 = __uint_as_float((m2 << 16) & 0x7FFF0000u), m1 = __uint_as_float(m2 & 0x7FFF0000u);
+        sb0 = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(m0) : e8m0_scale(m0, round);
+        sb1 = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(m1) : e8m0_scale(m1, round);
+        const float2 inv = make_float2(inv_scale(sb0), inv_scale(sb1));
+#pragma unroll
+        for (int r = 0; r < 32; r += 4) {
+            float2 q[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) q[i] = mul2(bf16x2_to_f32x2(xr[r + i]), inv);
+            out0[r / 4] = cvt_fp8x4<ELEM>(q[0].x, q[1].x, q[2].x, q[3].x);
+            out1[r / 4] = cvt_fp8x4<ELEM>(q[0].y, q[1].y, q[2].y, q[3].y);
+        }
+        return;
+    }
     float m0 = 0.f, m1 = 0.f;
 #pragma unroll
     for (int r = 0; r < 32; r += 4) {

@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_
 // token block) leave as one 4-byte store.
 constexpr int kToCols = 64, kToTokens = 128, kToThreads = 128, kToInBytes = kToTokens * kToCols * 2, kToOutBytes = kToCols * kToTokens;
 
-template <bool PAPER, int ELEM, bool ZSPILL>
+template <bool PAPER, int ELEM, bool ZSPILL, bool RHO>
 __global__ void __launch_bounds__(kToThreads, MXN_TO_MINB) cast_transposed_tile_kernel(const TransposedParams P)
 {
     extern __shared__ __align__(128) uint8_t tile_raw[];
@@ -266,9 +266,9 @@ __global__ void __launch_bounds__(kToThreads, MXN_TO_MINB) cast_transposed_tile_
         else asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" :: "r"(dst), "r"(0u) : "memory");
     }
     cp_async_commit();
-    {
+    if (RHO) {
         float rho = 1.0f;
-        if (P.rms != nullptr && tid < nblocks * 32) rho = recip_sat(__fadd_rn(P.rms[tbase + tid], P.eps));
+        if (tid < nblocks * 32) rho = recip_sat(__fadd_rn(P.rms[tbase + tid], P.eps));
         rho_s[warp][lane] = rho;
     }
     cp_async_wait<0>();
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(kToThreads, MXN_TO_MINB) cast_transposed_tile_
 #pragma unroll
         for (int r = 0; r < 32; ++r) asm volatile("ld.shared.b32 %0, [%1];" : "=r"(xr[r]) : "r"(wordaddr + (uint32_t)r * (kToCols * 2)));
         uint32_t o0[8], o1[8], sb0, sb1;
-        quantise_column_pair<PAPER, ELEM>(xr, rho_s[warp], P.round, o0, o1, sb0, sb1);
+        quantise_column_pair<PAPER, ELEM, RHO>(xr, rho_s[warp], P.round, o0, o1, sb0, sb1);
         // image rows 2*lane and 2*lane+1, bytes [32 warp, 32 warp + 32): chunks 2 warp and 2 warp + 1, swizzled by lane % 8
         const uint32_t r0 = out0 + (uint32_t)(2 * lane) * kToTokens, sw = (uint32_t)(lane & 7);
 #pragma unroll
@@ -348,9 +348,15 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
         const int64_t sx = (P.D + kToCols - 1) / kToCols, sy = (P.T + kToTokens - 1) / kToTokens;
         if ((sy + kMaxGridY - 1) / kMaxGridY <= 65535) {
             const bool zs = sy > kMaxGridY;
-            auto kfn = P.elem == ELEM_E5M2 ? (zs ? cast_transposed_tile_kernel<true, 2, true> : cast_transposed_tile_kernel<true, 2, false>)
-                       : P.round == MXN_ROUND_RCEIL_POW2 ? (zs ? cast_transposed_tile_kernel<true, 0, true> : cast_transposed_tile_kernel<true, 0, false>)
-                                                         : (zs ? cast_transposed_tile_kernel<false, 0, true> : cast_transposed_tile_kernel<false, 0, false>);
+            const bool rho = P.rms != nullptr;      // without a normaliser (e.g. the upstream gradient): the cheaper column phase
+            void (*kfn)(const TransposedParams);
+            if (P.elem == ELEM_E5M2) kfn = zs ? cast_transposed_tile_kernel<true, 2, true, false> : cast_transposed_tile_kernel<true, 2, false, false>;
+            else if (P.round == MXN_ROUND_RCEIL_POW2)
+                kfn = rho ? (zs ? cast_transposed_tile_kernel<true, 0, true, true> : cast_transposed_tile_kernel<true, 0, false, true>)
+                          : (zs ? cast_transposed_tile_kernel<true, 0, true, false> : cast_transposed_tile_kernel<true, 0, false, false>);
+            else
+                kfn = rho ? (zs ? cast_transposed_tile_kernel<false, 0, true, true> : cast_transposed_tile_kernel<false, 0, false, true>)
+                          : (zs ? cast_transposed_tile_kernel<false, 0, true, false> : cast_transposed_tile_kernel<false, 0, false, false>);
             const int smem = kToInBytes + kToOutBytes;
             const cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
             if (e != cudaSuccess) return e;
