@@ -398,7 +398,8 @@ def main():
         "ms_per_step_spread": spread(reps),
         "event_between_launches_ms_per_step": ms_serial,
         "tokens_per_s": T * world / (ms * 1e-3),
-        "gpu_launches": args.steps,
+        "gpu_launches": args.steps,                      # per timed region (ms_per_step is the median region)
+        "gpu_launches_all_regions": args.steps * REPEATS,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": gbs_one, "peak": peak, "unit": "GB/s", "frac": gbs_one / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_8TBs": gbs_one / 8000.0,
