@@ -23,6 +23,9 @@ namespace mxn {
 // warps of a CTA whose rows each span WPR warps
 __host__ __device__ constexpr int rows_per_cta(int wpr) { return MXN_FWD_WARPS / wpr > 1 ? MXN_FWD_WARPS / wpr : 1; }
 __host__ __device__ constexpr int cta_warps(int wpr) { return wpr * rows_per_cta(wpr); }
+// occupancy hint: the four-warp CTAs of the kernels without gain fit 64 registers per thread, i.e. 8 CTAs per SM
+// (one register more costs a whole CTA per SM: 7 instead of 8)
+__host__ __device__ constexpr int fwd_min_ctas(int wpr, bool gain) { return (cta_warps(wpr) == 4 && !gain) ? 8 : MXN_FWD_MIN_CTAS; }
 
 // ---- post-round estimator tables (appendix "Post-round MXNorm") ------------------------------------
 // f^-1 sampled at the 65 nodes 2^(i/64) of [1,2] for each block size, with the slope of every interval;
