@@ -140,7 +140,15 @@ def time_repeated(fn, n_sets: int, steps: int, warmup: int, stream, repeats: int
     return sorted(out)
 
 
+REST_S = 0.5        # idle time before a secondary kernel is timed (see time_median)
+
+
 def time_median(fn, n_sets: int, steps: int, warmup: int, stream, repeats: int = 3) -> float:
+    """Median of `repeats` timed regions, started from a rested GPU like the headline's regions are: on this pool a
+    kernel timed a second or more into an uninterrupted load runs up to 8 % slower than in a burst (power management;
+    the SM clock samples stay at their maximum), and the copy bandwidth the fractions refer to is a burst figure too."""
+    torch.cuda.synchronize()
+    time.sleep(REST_S)
     return statistics.median(time_repeated(fn, n_sets, steps, warmup, stream, repeats))
 
 
@@ -389,7 +397,9 @@ def main():
         "config": {"workload": workload_name(T, D),
                    "l2": f"inputs/outputs rotate over {SETS} buffer sets ({SETS * nbytes / 1e6:.0f} MB > 126 MB L2)",
                    "timing": f"{REPEATS} timed regions of {args.steps} launches each after {args.warmup} warm-up launches; ms_per_step "
-                             "is the median region, ms_per_step_spread its minimum and maximum; the other kernels: median of 3 regions",
+                             "is the median region, ms_per_step_spread its minimum and maximum; the other kernels: median of 3 regions, each kernel "
+                             f"after {REST_S} s of idle (burst figures, like the measured copy peak; seconds into an uninterrupted load "
+                             "the instruction-heavier kernels run up to 8 % slower on this pool)",
                    "launch": "back-to-back launches in one stream, as the library issues them: programmatic stream "
                              "serialisation (each kernel waits for the previous one before it reads or writes any value; launch "
                              "latency and L2 prefetch hints for the first-wave rows overlap the previous kernel's tail); "
@@ -524,10 +534,15 @@ def main():
             others["mxnorm_bwd_dx_only"] = {"ms": msbx, "gbs": (3 * T * D * 2 + 4 * T) / msbx / 1e6}
             del xb, gb, dxb
 
+        sampler2 = ClockSampler(local_rank)    # the secondary kernels run minutes into a sustained load: record the clock they saw
+        if rank == 0:
+            sampler2.start()
         try:   # context only: a failure here must not cost the headline line
             time_secondary_kernels()
         except Exception as e:   # noqa: BLE001
             result["others_error"] = f"{type(e).__name__}: {e}"[:300]
+        if rank == 0:
+            result["others_clocks"] = sampler2.stop()
         for v in others.values():
             v["frac_of_peak"] = v["gbs"] / peak
         result["others"] = others

@@ -15,7 +15,8 @@ HEADERS = ["mxn_device.cuh", "mxn_internal.h", "mxn_row.cuh", "mxn_col.cuh", os.
 # power-of-two products.
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "--ftz=false", "--prec-div=true", "--prec-sqrt=true",
-              "--split-compile", "0",   # the many template instantiations compile in parallel
+              # no --split-compile: it shortens the build of the forward kernels' file by a third, but changed the code
+              # generated for the backward kernel (two registers more, 64.4 -> 68.8 us at [16384, 4096])
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
 
 

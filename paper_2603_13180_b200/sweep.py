@@ -19,6 +19,7 @@ import argparse
 import json
 import math
 import os
+import time
 
 import torch
 
@@ -54,6 +55,10 @@ def _time(fn, sets, steps, warmup, stream, graph=True):
         b.record(stream)
     torch.cuda.synchronize()
     return a.elapsed_time(b) / steps * 1e3   # microseconds
+
+
+REST_S = 0.25   # idle time before each case: every case is a burst measurement (like the measured copy peak), not a
+                # point in one long uninterrupted load, which on this pool runs the same kernels up to 8 % slower
 
 
 def run(tokens, hidden, blocks, steps=30, warmup=5, l2_bytes=126 << 20, elem="e4m3", graph=True):
@@ -113,6 +118,8 @@ def _run(stream, tokens, hidden, blocks, steps, warmup, l2_bytes, elem, graph):
                                              0, mx.SCALES_SWIZZLE_128x4, sh)
                     assert st == 0, mx.status_string(st)
 
+                torch.cuda.synchronize()
+                time.sleep(REST_S)
                 t_mx = min(_time(mxn, sets, steps, warmup, stream, graph) for _ in range(2))
                 t_rms = min(_time(rms, sets, steps, warmup, stream, graph) for _ in range(2))
                 # yardstick: an elementwise copy kernel over per_set / 2 bytes (it reads and writes them: per_set bytes of
