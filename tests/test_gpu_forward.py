@@ -223,6 +223,19 @@ def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
         gu.assert_exact(got, gu.run_ref(oracle, "cast_nvfp4", x, global_scale=gs), f"mx_cast_nvfp4 {T}x{D} g={gs}")
 
 
+def test_gain_is_applied_after_the_normaliser(binding, oracle):
+    """Rows on which (x * rho~) * gamma and (x * gamma) * rho~ round to different E4M3 codes (found by search; the CPU pin of
+    the oracle uses the same rows): the kernels must take the first order, for MXNorm and for the conventional path."""
+    xb = np.zeros((3, 32), np.uint16)
+    xb[:, 0] = wl.f32_to_bf16_bits(np.array([2.5, 2.5, 5.0], np.float32))
+    xb[:, 1] = wl.f32_to_bf16_bits(np.array([-1.125, 0.28125, -0.5625], np.float32))
+    gb = np.full(32, 0x3F80, np.uint16)
+    gb[1] = wl.f32_to_bf16_bits(np.array([0.7265625], np.float32))[0]
+    got = gu.run_fwd(binding, oracle, "mx", xb, gb)
+    gu.assert_exact(got, gu.run_ref(oracle, "mx", xb, gb), "gain order")
+    assert list(got[0][:, 1]) == [229, 85, 213]
+
+
 def test_power_of_two_shift_on_gpu(binding, oracle):
     x, _ = rows(64, 1024, seed=23)
     xv = (x.astype(np.uint32) << 16).view(np.float32)
