@@ -3,11 +3,12 @@
 // (grad W = MXCast(grad H^T) MXCast(rho~ X) gamma: the activation is re-quantised along the token axis from
 // the cached X and rho~, the upstream gradient along its token axis as well).
 //
-// Work decomposition: a warp owns a tile of 32 tokens x 128 columns; a lane owns 4 columns and walks the
-// 32 rows (8-byte loads, a warp reads 256 contiguous bytes per row), so a column block's absmax needs no
-// cross-lane traffic and its 32 codes leave as one 32-byte store into row c of the transposed output.
-// The 4 warps of a CTA take 4 consecutive token tiles of the same columns, so each output row receives
-// 128 contiguous bytes per CTA.  Every input byte is read once, every output byte written once.
+// Two kernels.  The tile kernel (further down; D % 8 == 0 and a 16-byte aligned input) stages 128 tokens x 64 columns
+// in shared memory, quantises column pairs from there and writes the transposed tile in whole 128-byte lines.
+// The register kernel right below serves every other valid input (D % 4 == 0, 8-byte aligned): a warp owns a tile of
+// 32 tokens x 128 columns; a lane owns 4 columns and walks the 32 rows (8-byte loads, a warp reads 256 contiguous
+// bytes per row), so a column block's absmax needs no cross-lane traffic and its 32 codes leave as one 32-byte store
+// into row c of the transposed output.  Every input byte is read once, every output byte written once.
 #include "mxn_device.cuh"
 #include "mxn_internal.h"
 #include "mxn_col.cuh"
@@ -130,28 +131,6 @@ __global__ void __launch_bounds__(128) cast_transposed_kernel(const TransposedPa
     }
 }
 
-// ---- shared-memory staged variant (D % 8 == 0) ----------------------------------------------------
-// A CTA of 2 warps takes a tile of 32 tokens x 128 columns: the 32 row segments of 256 bytes arrive with
-// 16-byte cp.async copies (fully coalesced, no registers held while they fly), then a lane owns two
-// adjacent columns and walks the 32 rows through shared memory (consecutive lanes read consecutive words:
-// conflict-free).  A CTA processes MXN_TR_TPC consecutive token tiles of the same columns with two stages,
-// so the next tile streams in while the current one is quantised.
-#ifndef MXN_TR_TPC
-#define MXN_TR_TPC 1   // token tiles per CTA (measured at [16384,4096]: 1 -> 39.0 us, 2 -> 49.2, 4 -> 47.5)
-#endif
-#ifndef MXN_TR_MINB
-#define MXN_TR_MINB 12
-#endif
-#ifndef MXN_TO_MINB
-#define MXN_TO_MINB 7   // resident CTAs per SM aimed for (measured at [16384,4096]: 5 -> 35.1 us, 6 -> 32.9, 7 -> 32.0, 8 spills -> 40.1)
-#endif
-constexpr int kTsStages = MXN_TR_TPC > 1 ? 2 : 1;
-#ifndef MXN_TR_COLS
-#define MXN_TR_COLS 128   // columns per CTA tile, 64 per warp (measured at [16384,4096]: 64 -> 36.4 us, 128 -> 34.1, 256 -> 36.0, 512 -> 40.7, 1024 -> 54.2)
-#endif
-constexpr int kTsCols = MXN_TR_COLS, kTsThreads = kTsCols / 2, kTsRowBytes = kTsCols * 2, kTsStageBytes = 32 * kTsRowBytes,
-              kTsTpc = MXN_TR_TPC, kTsChunksPerRow = kTsRowBytes / 16, kTsChunksPerThread = 32 * kTsChunksPerRow / kTsThreads;
-
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(src) : "memory");
@@ -160,71 +139,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-template <bool PAPER, int ELEM, bool ZSPILL>
-__global__ void __launch_bounds__(kTsThreads, MXN_TR_MINB) cast_transposed_smem_kernel(const TransposedParams P)
-{
-    extern __shared__ __align__(128) uint8_t tile_raw[];
-    __shared__ __align__(16) float rho_s[2][32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t tile0 = (uint32_t)__cvta_generic_to_shared(tile_raw);
-    const int ctile = blockIdx.x * kTsCols;                  // first column of the CTA's tile
-    const int64_t tbase = (int64_t)token_tile_index<ZSPILL>() * kTsTpc * 32;   // first token of the CTA
-    {   // the first tile into L2 before the wait for the previous kernel (a hint: see prefetch_l2_bulk): one 128-byte line per thread
-        const int row = tid / (kTsRowBytes / 128), part = tid % (kTsRowBytes / 128);
-        const bool first_wave = (uint64_t)token_tile_index<ZSPILL>() * gridDim.x < 148u * 16u;   // later CTAs start after the wait is over
-        if (first_wave && row < 32 && tbase + row < P.T && ctile + part * 64 < P.D)
-            asm volatile("prefetch.global.L2 [%0];" :: "l"(P.x + (tbase + row) * P.D + ctile + part * 64) : "memory");
-    }
-    pdl_prologue();
-
-    auto issue = [&](int tt) {
-        const int64_t t0 = tbase + (int64_t)tt * 32;
-        const uint32_t stage = tile0 + (uint32_t)(tt & 1) * kTsStageBytes;
-        if (t0 < P.T) {
-#pragma unroll
-            for (int i = 0; i < kTsChunksPerThread; ++i) {
-                const int id = i * kTsThreads + tid, row = id / kTsChunksPerRow, c16 = id % kTsChunksPerRow;
-                const int col = ctile + c16 * 8;
-                const uint32_t dst = stage + (uint32_t)row * kTsRowBytes + (uint32_t)c16 * 16;
-                if (col < P.D) cp_async16(dst, P.x + (t0 + row) * P.D + col);
-                else asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" :: "r"(dst), "r"(0u) : "memory");
-            }
-            if (tid < 32) {
-                float rho = 1.0f;
-                if (P.rms != nullptr) {
-                    rho = recip_sat(__fadd_rn(P.rms[t0 + tid], P.eps));
-                }
-                rho_s[tt & 1][tid] = rho;
-            }
-        }
-        cp_async_commit();
-    };
-
-    issue(0);
-#pragma unroll 1
-    for (int tt = 0; tt < kTsTpc; ++tt) {
-        const int64_t t0 = tbase + (int64_t)tt * 32;
-        if (t0 >= P.T) break;                       // uniform over the CTA
-        if (tt + 1 < kTsTpc) issue(tt + 1);
-        else cp_async_commit();                     // keeps the group count uniform
-        cp_async_wait<1>();
-        __syncthreads();
-
-        const uint32_t stage = tile0 + (uint32_t)(tt & 1) * kTsStageBytes;
-        const float* rho = rho_s[tt & 1];
-        const uint32_t wordaddr = stage + (uint32_t)(warp * 32 + lane) * 4;
-        uint32_t xr[32];
-#pragma unroll
-        for (int r = 0; r < 32; ++r) asm volatile("ld.shared.b32 %0, [%1];" : "=r"(xr[r]) : "r"(wordaddr + (uint32_t)r * kTsRowBytes));
-
-        uint32_t out0[8], out1[8], sb0, sb1;
-        quantise_column_pair<PAPER, ELEM>(xr, rho, P.round, out0, out1, sb0, sb1);
-        const int c = ctile + (warp * 32 + lane) * 2;
-        if (c < P.D) store_column_pair(P.codes, P.scales, P.T, P.KT, P.tiles_per_row, P.layout, c, t0, out0, out1, sb0, sb1);
-        __syncthreads();   // the stage may be refilled by the next issue()
-    }
-    cp_async_wait<0>();
-}
+#ifndef MXN_TO_MINB
+#define MXN_TO_MINB 7   // resident CTAs per SM aimed for (measured at [16384,4096]: 5 -> 35.1 us, 6 -> 32.9, 7 -> 32.0, 8 spills -> 40.1)
+#endif
 
 // ---- output-staged variant (D % 8 == 0, x 16-byte aligned) ------------------------------------------
 // A CTA of 4 warps takes a tile of 128 tokens x 64 columns.  The 128 row segments of 128 bytes arrive with 16-byte
@@ -342,7 +259,6 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#ifndef MXN_TR_NO_TILE
     // 16-byte row chunks need D % 8 == 0 and a 16-byte aligned base (then every row start is 16-byte aligned)
     if (P.D % 8 == 0 && (reinterpret_cast<uintptr_t>(P.x) & 15) == 0) {
         const int64_t sx = (P.D + kToCols - 1) / kToCols, sy = (P.T + kToTokens - 1) / kToTokens;
@@ -366,25 +282,6 @@ cudaError_t launch_cast_transposed(TransposedParams P, cudaStream_t stream)
             return cudaLaunchKernelEx(&cfg, kfn, P);
         }
     }
-#endif
-#ifndef MXN_TR_NO_SMEM
-    if (P.D % 8 == 0 && (reinterpret_cast<uintptr_t>(P.x) & 15) == 0) {   // 16-byte row chunks: the shared-memory staged kernel
-        const int64_t sx = (P.D + kTsCols - 1) / kTsCols, sy = (P.T / 32 + kTsTpc - 1) / kTsTpc;
-        if ((sy + kMaxGridY - 1) / kMaxGridY <= 65535) {
-            const bool zs = sy > kMaxGridY;
-            auto kfn = P.elem == ELEM_E5M2 ? (zs ? cast_transposed_smem_kernel<true, 2, true> : cast_transposed_smem_kernel<true, 2, false>)
-                       : P.round == MXN_ROUND_RCEIL_POW2 ? (zs ? cast_transposed_smem_kernel<true, 0, true> : cast_transposed_smem_kernel<true, 0, false>)
-                                                         : (zs ? cast_transposed_smem_kernel<false, 0, true> : cast_transposed_smem_kernel<false, 0, false>);
-            const int smem = kTsStages * kTsStageBytes;
-            const cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            cfg.gridDim = token_tile_grid(sx, sy);
-            cfg.blockDim = dim3(kTsThreads);
-            cfg.dynamicSmemBytes = smem;
-            return cudaLaunchKernelEx(&cfg, kfn, P);
-        }
-    }
-#endif
     const bool zs = gy > kMaxGridY;
     auto kfn = P.elem == ELEM_E5M2 ? (zs ? cast_transposed_kernel<true, 2, true> : cast_transposed_kernel<true, 2, false>)
                : P.round == MXN_ROUND_RCEIL_POW2 ? (zs ? cast_transposed_kernel<true, 0, true> : cast_transposed_kernel<true, 0, false>)
