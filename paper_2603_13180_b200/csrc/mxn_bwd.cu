@@ -80,9 +80,17 @@ constexpr int kBwdMaxStages = 8;
 #define MXN_BWD_CTAS 2           // resident CTAs per SM the register allocator and the ring size aim for
 #endif
 
+// resident CTAs per SM the register allocator is asked to make room for: CTAs of at most 192 threads (short rows, or
+// one vector per thread) need few registers and little shared memory, and only more CTAs per SM give short rows enough
+// rows in flight
+__host__ __device__ constexpr int bwd_ctas_per_sm(int V, int NT) { return NT > MXN_BWD_THREADS ? 1 : (V == 1 || NT <= 192) ? 3 : MXN_BWD_CTAS; }
+
 template <int V, int NT, bool GAIN, bool DGAIN>
-__global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) bwd_kernel(const BwdParams P)
+__global__ void __launch_bounds__(NT, bwd_ctas_per_sm(V, NT)) bwd_kernel(const BwdParams P)
 {
+    // four vectors per thread with gain and gain gradient do not fit 128 registers if t = g/r*gamma is kept between the
+    // two phases of a row: that variant recomputes it (the same operations, hence the same bits)
+    constexpr bool KEEP_T = !(V == 4 && GAIN && DGAIN);
     extern __shared__ __align__(128) uint8_t ring_raw[];
     __shared__ uint64_t full[kBwdMaxStages];
     __shared__ float red[2][16];
@@ -158,7 +166,7 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
         //   dgamma += x*gi ;  dot += t*x  (= sum_d h x / r) ;  later  dX = t - x * (dot/(D r^2)).
         // (two elements per instruction: packed binary32 multiply and fused multiply-add, each half an
         //  ordinary IEEE operation)
-        float2 tt[V][4];
+        float2 tt[KEEP_T ? V : 1][4];
         float2 dd = make_float2(0.f, 0.f);
         const float2 inv_r2 = make_float2(inv_r, inv_r);
 #pragma unroll
@@ -171,7 +179,7 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
                 const float2 gi = mul2(bf16x2_to_f32x2(ga[j]), inv_r2);
                 if (DGAIN) acc[v][j] = __ffma2_rn(x2, gi, acc[v][j]);
                 const float2 t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gam[v][j])) : gi;
-                tt[v][j] = t2;
+                if (KEEP_T) tt[v][j] = t2;
                 dd = __ffma2_rn(t2, x2, dd);
             }
         }
@@ -215,10 +223,20 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
             const int vi = tid + v * n;
             if (vi >= nvec) continue;
             const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
+            const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
             float2 o[4];
             const float2 nc2 = make_float2(-c2, -c2);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) o[j] = __ffma2_rn(bf16x2_to_f32x2(xa[j]), nc2, tt[v][j]);
+            for (int j = 0; j < 4; ++j) {
+                float2 t2;
+                if (KEEP_T) {
+                    t2 = tt[v][j];
+                } else {
+                    const float2 gi = mul2(bf16x2_to_f32x2(ga[j]), inv_r2);
+                    t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gam[v][j])) : gi;
+                }
+                o[j] = __ffma2_rn(bf16x2_to_f32x2(xa[j]), nc2, t2);
+            }
             if (P.dx_is_fp32) {
                 float* dp = static_cast<float*>(P.dx) + row * P.D + (int64_t)vi * 8;
                 st_v4(dp, reinterpret_cast<const uint32_t*>(&o[0]));
@@ -251,7 +269,7 @@ __global__ void __launch_bounds__(NT, NT > MXN_BWD_THREADS ? 1 : MXN_BWD_CTAS) b
 // then the 32 warp sums are added 0..31.  Launched with programmatic stream serialisation so that its
 // launch latency hides behind the tail of the main kernel; it waits for the main kernel's results
 // before the first load.
-constexpr int kReduceMaxRowsPerWarp = 10;   // 32 warps x 10 rows >= 296 partial rows
+constexpr int kReduceMaxRowsPerWarp = 10;   // loads a warp keeps in flight: 32 warps x 10 rows >= the 296 partial rows of wide rows
 
 __global__ void __launch_bounds__(1024) bwd_dgain_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dgain,
                                                                int D, int parts)
@@ -260,17 +278,17 @@ __global__ void __launch_bounds__(1024) bwd_dgain_reduce_kernel(const float* __r
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int col = blockIdx.x * 32 + lane;
     pdl_prologue();
-    float v[kReduceMaxRowsPerWarp];
+    float a = 0.0f;
+    for (int base = warp; base < parts; base += 32 * kReduceMaxRowsPerWarp) {   // one batch covers 320 partial rows
+        float v[kReduceMaxRowsPerWarp];
 #pragma unroll
-    for (int i = 0; i < kReduceMaxRowsPerWarp; ++i) {
-        const int p = warp + 32 * i;
-        v[i] = (col < D && p < parts) ? partial[(int64_t)p * D + col] : 0.0f;
+        for (int i = 0; i < kReduceMaxRowsPerWarp; ++i) {
+            const int p = base + 32 * i;
+            v[i] = (col < D && p < parts) ? partial[(int64_t)p * D + col] : 0.0f;
+        }
+#pragma unroll
+        for (int i = 0; i < kReduceMaxRowsPerWarp; ++i) a += v[i];
     }
-    float a = v[0];
-#pragma unroll
-    for (int i = 1; i < kReduceMaxRowsPerWarp; ++i) a += v[i];
-    if (col < D)
-        for (int p = warp + 32 * kReduceMaxRowsPerWarp; p < parts; p += 32) a += partial[(int64_t)p * D + col];   // more rows than expected
     s[warp][lane] = a;
     __syncthreads();
     if (warp == 0 && col < D) {
@@ -284,21 +302,40 @@ __global__ void __launch_bounds__(1024) bwd_dgain_reduce_kernel(const float* __r
 // threads per CTA, vectors per thread, ring stages and CTAs per SM for a row of D elements
 struct BwdPlan { int threads, V, stages, stage_bytes, ctas_per_sm; size_t smem; };
 
-static bool plan_bwd(int64_t D, BwdPlan* pl)
+// Threads per CTA, vectors per thread and CTAs per SM for rows of D elements.  Measured at 16384 rows:
+//   D <= 2048: two vectors per thread in narrow CTAs and many of them (D = 2048: 128 threads x 5-6 CTAs per SM 36.1 / 29.5 us
+//   with / without the gain gradient, against 45.4 / 38.1 us for 256 threads x 3; D = 1536: 96 x 6-8: 30.6 / 23.9 against
+//   42.3 / 34.0; D = 1024: 64 x 8-12: 28.4 / 16.9 against 30.3 / 28.1 for 128 x 4).  The count follows the registers of the
+//   variant (20 or 24 warps per SM); with the gain gradient at most 8 CTAs, because every CTA adds a row of partial sums.
+//   D = 3072: 192 threads x 3 CTAs (49.7 / 44.3 us; 4 CTAs: 64.7 / 45.8).  D = 4096: 256 x 2 (65.2 / 59.2; 3 CTAs: 82.4 / 62.4).
+//   Wider rows: 3 or 4 vectors per thread, 2 CTAs per SM; beyond 8192 elements 512 threads, 1 CTA.
+static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl)
 {
     if (D <= 0 || D % 8 != 0 || D > 16384) return false;
     const int64_t nvec = D / 8;
-    int n = (int)(((nvec < MXN_BWD_THREADS ? nvec : MXN_BWD_THREADS) + 31) / 32 * 32);
-    int v = (int)((nvec + n - 1) / n);
-    if (v > 4) {   // wide rows: more threads before more vectors per thread
-        n = 512;
+    int n, v, ctas;
+    if (nvec <= 256) {
+        v = nvec > 32 ? 2 : 1;
+        n = (int)(((nvec + v - 1) / v + 31) / 32 * 32);
+        const int warps = n / 32;
+        ctas = dgain ? 20 / warps : 24 / warps;
+        const int cap = dgain ? 8 : 12;
+        ctas = ctas > cap ? cap : ctas;
+    } else {
+        n = MXN_BWD_THREADS;
         v = (int)((nvec + n - 1) / n);
+        if (v > 4) {   // wide rows: more threads before more vectors per thread
+            n = 512;
+            v = (int)((nvec + n - 1) / n);
+        }
+        if (v > 4) return false;
+        n = (int)(((nvec + v - 1) / v + 31) / 32 * 32);          // no more threads than v vectors each need (D = 3072: 192, not 256)
+        ctas = n > MXN_BWD_THREADS ? 1 : (v == 2 && n <= 192) ? 3 : MXN_BWD_CTAS;
     }
-    if (v > 4) return false;
     pl->threads = n;
-    pl->V = v <= 2 ? v : 4;
+    pl->V = v;                                                   // 1..4, each instantiated
+    pl->ctas_per_sm = ctas;
     pl->stage_bytes = 2 * (int)((D * 2 + 127) / 128 * 128);     // x row + g row
-    pl->ctas_per_sm = n <= MXN_BWD_THREADS ? MXN_BWD_CTAS : 1;
     const int budget = 200 * 1024 / pl->ctas_per_sm;            // shared memory per CTA
     int st = budget / pl->stage_bytes;
     pl->stages = st < 2 ? 2 : (st > kBwdMaxStages ? kBwdMaxStages : st);
@@ -309,13 +346,13 @@ static bool plan_bwd(int64_t D, BwdPlan* pl)
 bool bwd_shape_supported(int64_t D)
 {
     BwdPlan pl;
-    return plan_bwd(D, &pl);
+    return plan_bwd(D, true, &pl);
 }
 
 int bwd_parts(int64_t T, int64_t D)
 {
     BwdPlan pl;
-    if (!plan_bwd(D, &pl)) return 0;
+    if (!plan_bwd(D, true, &pl)) return 0;      // the plan with the gain gradient: the one that needs the workspace
     const int64_t cap = (int64_t)kSMs * pl.ctas_per_sm;
     return (int)(T < cap ? (T < 1 ? 1 : T) : cap);
 }
@@ -333,15 +370,20 @@ static bwd_fn pick_bwd(bool gain, bool dgain)
 
 cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
 {
+    const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
     BwdPlan pl;
-    if (!plan_bwd(P.D, &pl)) return cudaErrorInvalidValue;
+    if (!plan_bwd(P.D, dgain, &pl)) return cudaErrorInvalidValue;
     P.stages = pl.stages;
     P.stage_bytes = pl.stage_bytes;
-    const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
+    {   // the grid of this variant (with the gain gradient it equals bwd_parts(T, D), which sized the workspace)
+        const int64_t cap = (int64_t)kSMs * pl.ctas_per_sm;
+        P.parts = (int)(P.T < cap ? P.T : cap);
+    }
     bwd_fn fn;
     if (pl.threads > MXN_BWD_THREADS) fn = pick_bwd<4, 512>(gain, dgain);
     else if (pl.V == 1) fn = pick_bwd<1, MXN_BWD_THREADS>(gain, dgain);
-    else if (pl.V == 2) fn = pick_bwd<2, MXN_BWD_THREADS>(gain, dgain);
+    else if (pl.V == 2) fn = pl.threads <= 192 ? pick_bwd<2, 192>(gain, dgain) : pick_bwd<2, MXN_BWD_THREADS>(gain, dgain);   // 192: registers for 3+ CTAs per SM
+    else if (pl.V == 3) fn = pick_bwd<3, MXN_BWD_THREADS>(gain, dgain);
     else fn = pick_bwd<4, MXN_BWD_THREADS>(gain, dgain);
     cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
