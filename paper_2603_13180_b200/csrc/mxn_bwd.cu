@@ -124,14 +124,21 @@ __global__ void __launch_bounds__(NT, bwd_ctas_per_sm(V, NT)) bwd_kernel(const B
         }
     }
 
-    uint32_t gam[V][4];   // gain kept as packed bf16 pairs
+    // gain as packed bf16 pairs: in registers, except in the variant that is short of them (KEEP_T false), which parks
+    // it in shared memory behind the ring and reads each vector back where it is used
+    uint32_t gam[KEEP_T ? V : 1][4];
+    const uint32_t gain_smem = ring + (uint32_t)stages * (uint32_t)P.stage_bytes;
     float2 acc[V][4];
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int vi = tid + v * n;
         uint4 gw = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);   // ones
         if (GAIN && vi < nvec) gw = __ldg(reinterpret_cast<const uint4*>(P.gain) + vi);
-        gam[v][0] = gw.x; gam[v][1] = gw.y; gam[v][2] = gw.z; gam[v][3] = gw.w;
+        if (KEEP_T) {
+            gam[v][0] = gw.x; gam[v][1] = gw.y; gam[v][2] = gw.z; gam[v][3] = gw.w;
+        } else if (vi < nvec) {
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" :: "r"(gain_smem + (uint32_t)vi * 16u), "r"(gw.x), "r"(gw.y), "r"(gw.z), "r"(gw.w) : "memory");
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[v][j] = make_float2(0.0f, 0.0f);
     }
@@ -173,12 +180,16 @@ __global__ void __launch_bounds__(NT, bwd_ctas_per_sm(V, NT)) bwd_kernel(const B
         for (int v = 0; v < V; ++v) {
             const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
             const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
+            uint4 gq = make_uint4(0, 0, 0, 0);
+            if (!KEEP_T && tid + v * n < nvec) gq = lds_v4(gain_smem + (uint32_t)(tid + v * n) * 16u);
+            const uint32_t gm[4] = {KEEP_T ? gam[KEEP_T ? v : 0][0] : gq.x, KEEP_T ? gam[KEEP_T ? v : 0][1] : gq.y,
+                                    KEEP_T ? gam[KEEP_T ? v : 0][2] : gq.z, KEEP_T ? gam[KEEP_T ? v : 0][3] : gq.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const float2 x2 = bf16x2_to_f32x2(xa[j]);
                 const float2 gi = mul2(bf16x2_to_f32x2(ga[j]), inv_r2);
                 if (DGAIN) acc[v][j] = __ffma2_rn(x2, gi, acc[v][j]);
-                const float2 t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gam[v][j])) : gi;
+                const float2 t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gm[j])) : gi;
                 if (KEEP_T) tt[v][j] = t2;
                 dd = __ffma2_rn(t2, x2, dd);
             }
@@ -224,6 +235,10 @@ __global__ void __launch_bounds__(NT, bwd_ctas_per_sm(V, NT)) bwd_kernel(const B
             if (vi >= nvec) continue;
             const uint32_t xa[4] = {xw[v].x, xw[v].y, xw[v].z, xw[v].w};
             const uint32_t ga[4] = {gw[v].x, gw[v].y, gw[v].z, gw[v].w};
+            uint4 gq = make_uint4(0, 0, 0, 0);
+            if (!KEEP_T) gq = lds_v4(gain_smem + (uint32_t)vi * 16u);
+            const uint32_t gm[4] = {KEEP_T ? gam[KEEP_T ? v : 0][0] : gq.x, KEEP_T ? gam[KEEP_T ? v : 0][1] : gq.y,
+                                    KEEP_T ? gam[KEEP_T ? v : 0][2] : gq.z, KEEP_T ? gam[KEEP_T ? v : 0][3] : gq.w};
             float2 o[4];
             const float2 nc2 = make_float2(-c2, -c2);
 #pragma unroll
@@ -233,7 +248,7 @@ __global__ void __launch_bounds__(NT, bwd_ctas_per_sm(V, NT)) bwd_kernel(const B
                     t2 = tt[v][j];
                 } else {
                     const float2 gi = mul2(bf16x2_to_f32x2(ga[j]), inv_r2);
-                    t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gam[v][j])) : gi;
+                    t2 = GAIN ? mul2(gi, bf16x2_to_f32x2(gm[j])) : gi;
                 }
                 o[j] = __ffma2_rn(bf16x2_to_f32x2(xa[j]), nc2, t2);
             }
@@ -312,7 +327,7 @@ struct BwdPlan { int threads, V, stages, stage_bytes, ctas_per_sm; size_t smem; 
 //   variant (20 or 24 warps per SM); with the gain gradient at most 8 CTAs, because every CTA adds a row of partial sums.
 //   D = 3072: 192 threads x 3 CTAs (49.7 / 44.3 us; 4 CTAs: 64.7 / 45.8).  D = 4096: 256 x 2 (65.2 / 59.2; 3 CTAs: 82.4 / 62.4).
 //   Wider rows: 3 or 4 vectors per thread, 2 CTAs per SM; beyond 8192 elements 512 threads, 1 CTA.
-static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl)
+static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false)
 {
     if (D <= 0 || D % 8 != 0 || D > 16384) return false;
     const int64_t nvec = D / 8;
@@ -327,11 +342,10 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl)
     } else {
         n = MXN_BWD_THREADS;
         v = (int)((nvec + n - 1) / n);
-        if (v > 4) {   // wide rows: more threads before more vectors per thread
-            n = 512;
-            v = (int)((nvec + n - 1) / n);
+        if (v > 4) {   // wide rows: up to 512 threads; that kernel exists with four vectors per thread only
+            if (nvec > 4 * 512) return false;
+            v = 4;
         }
-        if (v > 4) return false;
         n = (int)(((nvec + v - 1) / v + 31) / 32 * 32);          // no more threads than v vectors each need (D = 3072: 192, not 256)
         ctas = n > MXN_BWD_THREADS ? 1 : (v == 2 && n <= 192) ? 3 : MXN_BWD_CTAS;
     }
@@ -343,6 +357,11 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl)
     int st = budget / pl->stage_bytes;
     pl->stages = st < 2 ? 2 : (st > kBwdMaxStages ? kBwdMaxStages : st);
     pl->smem = (size_t)pl->stages * pl->stage_bytes;
+    if (pl->V == 4 && gain && dgain) {   // room behind the ring for the gain of the variant that parks it there
+        const size_t gain_bytes = (size_t)(D * 2 + 127) / 128 * 128;
+        while (pl->stages > 2 && (pl->smem + gain_bytes) * pl->ctas_per_sm > 216 * 1024) pl->smem = (size_t)(--pl->stages) * pl->stage_bytes;
+        pl->smem += gain_bytes;
+    }
     return pl->smem <= 220 * 1024;
 }
 
@@ -375,7 +394,7 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
 {
     const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
     BwdPlan pl;
-    if (!plan_bwd(P.D, dgain, &pl)) return cudaErrorInvalidValue;
+    if (!plan_bwd(P.D, dgain, &pl, gain)) return cudaErrorInvalidValue;
     P.stages = pl.stages;
     P.stage_bytes = pl.stage_bytes;
     {   // the grid of this variant (with the gain gradient it equals bwd_parts(T, D), which sized the workspace)
