@@ -401,6 +401,9 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
         const int64_t cap = (int64_t)kSMs * pl.ctas_per_sm;
         P.parts = (int)(P.T < cap ? P.T : cap);
     }
+    // the kernel template below must be the one the plan sized shared memory for (the four-vector variant with gain and
+    // gain gradient keeps the gain behind the ring): a mismatch is refused here instead of reaching the device
+    if ((pl.threads > MXN_BWD_THREADS ? 4 : pl.V) != pl.V || pl.threads * pl.V < P.D / 8) return cudaErrorInvalidValue;
     bwd_fn fn;
     if (pl.threads > MXN_BWD_THREADS) fn = pick_bwd<4, 512>(gain, dgain);
     else if (pl.V == 1) fn = pick_bwd<1, MXN_BWD_THREADS>(gain, dgain);
