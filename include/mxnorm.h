@@ -113,6 +113,18 @@ mxn_status mxn_selftest_bounded_wait(unsigned int polls, void* cuda_stream);
  * utility, not part of the hot path).  *mismatches_out receives the number of differing quotients (0). */
 mxn_status mxn_selftest_division(unsigned long long* mismatches_out);
 
+/* Diagnostics, host only (no device is touched): walks every row length D <= max_D that the forward entry points
+ * accept, for each block size, row statistic, element format, gain / residual option and scale rounding rule they can
+ * ask for, and counts the combinations for which the launcher would find no compiled kernel (expected: 0, i.e. a shape
+ * that passes the argument checks can always be launched).  *missing_out receives the count; when it is non-zero
+ * *first_D_out / *first_case_out (either may be NULL) receive the first such row length and a decimal code
+ * ((block * 10 + variant) * 10 + statistic) * 10 + rounding rule, with variant 0 E4M3, 1 E4M3 with gain, 2 E5M2,
+ * 3 MXFP4, 4 fused residual add, 5 NVFP4 and statistic 0 none, 1 RMS, 2 MX estimate, 3 post-round estimate.
+ * The walk also covers the backward: every row length it accepts, with and without gain and gain gradient, must have
+ * a launch plan whose kernel variant exists and whose shared memory fits (first case code -(1 + 2*gain + dgain)).
+ * Returns MXN_ERR_NULL when missing_out is NULL and MXN_ERR_SHAPE when max_D < 16. */
+mxn_status mxn_selftest_dispatch(int64_t max_D, long long* missing_out, int64_t* first_D_out, int* first_case_out);
+
 /* MXCast - Section 3.2 "Conversion to MXFP8", Eqs. S_tk = cast(m_tk / 256; E8M0),
  * V_tkb = cast(X_tkb / S_tk; E4M3).
  *   x_bf16 [T,D] in; codes_u8 [T,D] out; scales_u8 out (biased E8M0 exponents;

@@ -22,7 +22,7 @@ EXPORTS = ("mxn_scale_bytes", "mxn_status_string", "mx_cast", "rmsnorm_mxfp8_fwd
            "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_bwd_workspace_bytes", "mxnorm_fwd_host",
            "mxnorm_fwd_host_workspace_bytes", "mxnorm_bwd_noalloc", "mxnorm_bwd_noalloc_max_scratch_bytes",
            "mxn_device_timeouts", "mxn_device_timeouts_reset", "mxn_selftest_bounded_wait", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
-           "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
+           "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division", "mxn_selftest_dispatch",
            "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
            "mxnorm_add_fwd", "mx_cast_nvfp4")
 
@@ -46,6 +46,8 @@ lib.mxn_selftest_bounded_wait.argtypes = [ctypes.c_uint, _vp]
 lib.mxn_selftest_bounded_wait.restype = _i32
 lib.mxn_selftest_division.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
 lib.mxn_selftest_division.restype = _i32
+lib.mxn_selftest_dispatch.argtypes = [_i64, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(_i64), ctypes.POINTER(_i32)]
+lib.mxn_selftest_dispatch.restype = _i32
 lib.mx_cast.argtypes = [_vp, _i64, _i64, _i32, _vp, _vp, _i32, _i32, _vp]
 lib.rmsnorm_mxfp8_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
 lib.mxnorm_fwd.argtypes = [_vp, _vp, _i64, _i64, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _i32, _i32, _vp]
@@ -71,7 +73,7 @@ lib.mxnorm_bwd_noalloc_max_scratch_bytes.argtypes = []
 lib.mxnorm_bwd_noalloc_max_scratch_bytes.restype = _sz
 for _name in ("mx_cast", "rmsnorm_mxfp8_fwd", "mxnorm_fwd", "mxnorm_nvfp4_fwd", "mxnorm_bwd", "mxnorm_fwd_host",
               "mxnorm_bwd_noalloc", "mx_cast_fp4", "rmsnorm_mxfp4_fwd", "mxnorm_mxfp4_fwd",
-           "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division",
+           "mx_cast_transposed", "rmsnorm_nvfp4_fwd", "mxn_selftest_division", "mxn_selftest_dispatch",
            "mx_cast_e5m2", "mx_cast_transposed_e5m2", "mxnorm_postround_fwd",
            "mxnorm_add_fwd", "mx_cast_nvfp4"):
     getattr(lib, _name).restype = _i32
@@ -132,6 +134,14 @@ def selftest_division() -> int:
     n = ctypes.c_ulonglong(0)
     _check(lib.mxn_selftest_division(ctypes.byref(n)), "mxn_selftest_division")
     return int(n.value)
+
+
+def selftest_dispatch(max_D: int = 65536):
+    """Host only: (number of accepted forward shapes and options without a compiled kernel, first such D, its case
+    code); the count is expected to be 0."""
+    n, d, c = ctypes.c_longlong(0), _i64(0), _i32(0)
+    _check(lib.mxn_selftest_dispatch(max_D, ctypes.byref(n), ctypes.byref(d), ctypes.byref(c)), "mxn_selftest_dispatch")
+    return int(n.value), int(d.value), int(c.value)
 
 
 def scale_bytes(T: int, K: int, layout: int = SCALES_ROWMAJOR) -> int:

@@ -130,6 +130,29 @@ mxn_status mxn_selftest_division(unsigned long long* mismatches_out)
     return MXN_OK;
 }
 
+mxn_status mxn_selftest_dispatch(int64_t max_D, long long* missing_out, int64_t* first_D_out, int* first_case_out)
+{
+    if (missing_out == nullptr) return MXN_ERR_NULL;
+    if (max_D < 16) return MXN_ERR_SHAPE;
+    int64_t first_D = 0;
+    int first_case = 0;
+    int64_t missing = mxn::selftest_dispatch(max_D, &first_D, &first_case);
+    {
+        int64_t d = 0;
+        int c = 0;
+        const int64_t bad = mxn::selftest_bwd_plans(max_D, &d, &c);
+        if (missing == 0 && bad != 0) {
+            first_D = d;
+            first_case = c;
+        }
+        missing += bad;
+    }
+    *missing_out = (long long)missing;
+    if (first_D_out != nullptr) *first_D_out = first_D;
+    if (first_case_out != nullptr) *first_case_out = first_case;
+    return MXN_OK;
+}
+
 mxn_status mx_cast(const void* x_bf16, int64_t T, int64_t D, int block, void* codes_u8, void* scales_u8,
                    mxn_round round, mxn_scale_layout layout, void* cuda_stream)
 {

@@ -439,6 +439,36 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     return e;
 }
 
+// Host-only walk over every row length the backward accepts, with and without gain and gain gradient: counts the plans
+// the launcher would refuse or whose shared memory would not fit the CTAs per SM they ask for.  No device is touched.
+int64_t selftest_bwd_plans(int64_t max_D, int64_t* first_D, int* first_case)
+{
+    int64_t bad = 0;
+    for (int64_t D = 8; D <= max_D; D += 8) {
+        if (!bwd_shape_supported(D)) continue;
+        for (int c = 0; c < 4; ++c) {
+            const bool gain = (c & 2) != 0, dgain = (c & 1) != 0;
+            BwdPlan pl;
+            bool ok = plan_bwd(D, dgain, &pl, gain);
+            if (ok) {
+                const size_t ring = (size_t)pl.stages * pl.stage_bytes;
+                const size_t parked = pl.V == 4 && gain && dgain ? (size_t)(D * 2 + 127) / 128 * 128 : 0;
+                ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V == 4))
+                  && pl.threads % 32 == 0 && (int64_t)pl.threads * pl.V >= D / 8 && pl.stages >= 2 && pl.stages <= kBwdMaxStages
+                  && pl.stage_bytes >= 4 * D && pl.smem == ring + parked
+                  && pl.smem <= 227 * 1024                                             // one CTA's limit
+                  && (pl.smem + 2048) * pl.ctas_per_sm <= 228 * 1024                   // the SM's, with static and reserved bytes
+                  && pl.threads * pl.ctas_per_sm <= 2048;
+            }
+            if (!ok && bad++ == 0) {
+                *first_D = D;
+                *first_case = -(1 + c);
+            }
+        }
+    }
+    return bad;
+}
+
 cudaError_t read_timeouts(unsigned int* out)
 {
     return cudaMemcpyFromSymbol(out, g_bwd_timeouts, sizeof(unsigned int));

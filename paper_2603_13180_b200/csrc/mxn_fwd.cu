@@ -657,7 +657,9 @@ bool fwd_shape_supported(int64_t D, int B)
     return plan_row((int)(D / E), E, false, false, &wpr, &npass);   // the coarse set is the narrowest
 }
 
-cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
+// Everything a launch needs that does not depend on the pointers: the row plan written into P, the kernel, the grid and
+// the CTA size.  Kept apart from the launch so that the host-side self-test can walk every supported shape.
+static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out, int64_t* ctas_out, int* threads_out)
 {
     const bool mxfp4 = P.elem == ELEM_E2M1 && !nvfp4;
     const bool e5m2 = P.elem == ELEM_E5M2;
@@ -674,7 +676,7 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
                                 P.round == MXN_ROUND_RCEIL_POW2);
     P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
     P.chunks = nv_pair ? P.K / 2 : P.K * (B / E);
-    if (!plan_row(P.chunks, E, fine, nvfp4 && !nv_pair, &P.wpr, &P.npass)) return cudaErrorInvalidValue;
+    if (!plan_row(P.chunks, E, fine, nvfp4 && !nv_pair, &P.wpr, &P.npass)) return false;
     P.tiles_per_row = (P.K + 3) / 4;
     {
         const int count = stat == STAT_RMS ? P.D : P.K;   // divisor of the row statistic
@@ -686,19 +688,10 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     fwd_fn fn = nullptr;
     if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && (fine || mxfp4) && stat != STAT_POSTROUND) {
         fn = nvfp4 ? pick_multi_stat<2>(16, stat, rpw) : mxfp4 ? pick_multi_stat<1>(B, stat, rpw) : pick_multi_stat<0>(B, stat, rpw);
-        const int64_t rows_per_cta = (int64_t)MXN_FWD_WARPS * rpw;
-        const int64_t ctas = (P.T + rows_per_cta - 1) / rows_per_cta;
-        if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)ctas);
-        cfg.blockDim = dim3(MXN_FWD_WARPS * kWarp);
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, fn, P);
+        *fn_out = fn;
+        *ctas_out = (P.T + (int64_t)MXN_FWD_WARPS * rpw - 1) / ((int64_t)MXN_FWD_WARPS * rpw);
+        *threads_out = MXN_FWD_WARPS * kWarp;
+        return fn != nullptr;
     }
     if (nv_pair) fn = stat == STAT_RMS ? pick_nvfp4_pair<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4_pair<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4_pair<STAT_MX>(P.wpr, P.npass);
     else if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
@@ -709,14 +702,23 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     else if (B == 16) fn = pick_round<16, 1>(P.round, stat, has_gain, P.wpr, P.npass);
     else if (B == 32) fn = pick_round<32, 1>(P.round, stat, has_gain, P.wpr, P.npass);
     else fn = pick_round<32, 2>(P.round, stat, has_gain, P.wpr, P.npass);
-    if (fn == nullptr) return cudaErrorInvalidValue;
-    const int64_t ctas = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
-    if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    *fn_out = fn;
+    *ctas_out = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
+    *threads_out = warps * kWarp;
+    return fn != nullptr;
+}
+
+cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream)
+{
+    fwd_fn fn = nullptr;
+    int64_t ctas = 0;
+    int threads = 0;
+    if (!select_fwd(P, B, stat, nvfp4, &fn, &ctas, &threads) || ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
     // Programmatic stream serialisation: the kernel may be scheduled while the previous kernel of the
     // stream drains; it does not touch memory before that kernel has completed (pdl_prologue).
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas);
-    cfg.blockDim = dim3(warps * kWarp);
+    cfg.blockDim = dim3(threads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -724,6 +726,54 @@ cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t st
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fn, P);
+}
+
+// Host-only walk over every row length the shape check admits, in every combination of block size, statistic, element
+// format, gain, residual and rounding rule the entry points can ask for: counts the combinations for which no kernel is
+// instantiated (a launch would be refused) and reports the first.  No device is touched.
+int64_t selftest_dispatch(int64_t max_D, int64_t* first_D, int* first_case)
+{
+    int64_t missing = 0;
+    static const uint16_t dummy = 0;
+    for (int bi = 0; bi < 3; ++bi) {
+        const int B = 16 << bi;
+        for (int64_t D = B; D <= max_D; D += B) {
+            if (!fwd_shape_supported(D, B)) continue;
+            // every combination an entry point can ask for: variant 0 E4M3, 1 E4M3 with gain, 2 E5M2, 3 MXFP4,
+            // 4 residual add, 5 NVFP4; the scale rounding rule varies for the E4M3 variants only
+            for (int variant = 0; variant < 6; ++variant) {
+                for (int stat = 0; stat < 4; ++stat) {
+                    for (int round = 0; round <= MXN_ROUND_RCEIL_MAX; ++round) {
+                        const bool asked =
+                            variant == 0 ? (stat != STAT_POSTROUND || round == 0)
+                          : variant == 1 ? (stat == STAT_RMS || stat == STAT_MX)
+                          : variant == 2 ? (stat == STAT_NONE && round == 0)
+                          : variant == 3 ? (stat != STAT_POSTROUND && round == 0)
+                          : variant == 4 ? (stat == STAT_MX && round == 0)
+                                         : (B == 16 && stat != STAT_POSTROUND && round == 0);
+                        if (!asked) continue;
+                        FwdParams P = {};
+                        P.T = 1;
+                        P.D = (int)D;
+                        P.K = (int)(D / B);
+                        P.elem = variant == 2 ? ELEM_E5M2 : (variant == 3 || variant == 5) ? ELEM_E2M1 : ELEM_E4M3;
+                        P.gain = variant == 1 ? &dummy : nullptr;
+                        P.residual = variant == 4 ? &dummy : nullptr;
+                        P.round = round;
+                        fwd_fn fn = nullptr;
+                        int64_t ctas = 0;
+                        int threads = 0;
+                        if (select_fwd(P, B, stat, variant == 5, &fn, &ctas, &threads) && ctas == 1 && threads > 0) continue;
+                        if (missing++ == 0) {
+                            *first_D = D;
+                            *first_case = ((B * 10 + variant) * 10 + stat) * 10 + round;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    return missing;
 }
 
 // ---- host side of the post-round estimator: f, its inverse and the table --------------------------

@@ -33,6 +33,8 @@ struct FwdParams {
 bool fwd_shape_supported(int64_t D, int B);
 cudaError_t launch_fwd(FwdParams P, int B, int stat, bool nvfp4, cudaStream_t stream);
 cudaError_t selftest_division(unsigned long long* mismatches_host);
+int64_t selftest_dispatch(int64_t max_D, int64_t* first_D, int* first_case);   // host only
+int64_t selftest_bwd_plans(int64_t max_D, int64_t* first_D, int* first_case);  // host only
 cudaError_t postround_prepare(int B);   // uploads the f^-1 table for block size B to the current device (once)
 
 struct TransposedParams {

@@ -82,6 +82,16 @@ def test_argument_errors_are_statuses(binding):
     assert bwd(x=FAKE + 2) == 3 and bwd(ws=FAKE + 4) == 3
 
 
+def test_every_accepted_shape_has_a_kernel(binding):
+    # host-only walk of the launchers: every row length the argument checks admit, with every option an entry point can
+    # ask for, must select a compiled forward kernel, and every backward plan must fit the kernel it launches
+    missing, first_d, first_case = binding.selftest_dispatch(1 << 17)
+    assert missing == 0, (missing, first_d, first_case)
+    n = ctypes.c_longlong(7)
+    assert binding.lib.mxn_selftest_dispatch(8, ctypes.byref(n), None, None) == 2
+    assert binding.lib.mxn_selftest_dispatch(4096, None, None, None) == 1
+
+
 def test_binding_module_has_no_fallback():
     src = open(os.path.join(ROOT, "paper_2603_13180_b200", "binding.py")).read()
     assert "oracle" not in src.replace("CPU oracle", "")
