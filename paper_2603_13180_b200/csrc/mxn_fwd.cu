@@ -619,6 +619,9 @@ static fwd_fn pick_nvfp4_pair(int wpr, int npass)
 // splits that leave a lane little work when a row spans several warps (more warps, hence more synchronisation,
 // per row).  Measured at 16384 rows: D = 7168, B = 32: 4 warps x 2 passes at 87.5 % beat 7 warps x 1 pass at 100 %;
 // D = 2560, B = 16: 5 warps x 1 pass (16 elements per lane) at 100 % lost to 2 warps x 4 passes at 62.5 %.
+// Measured at 32768 rows, every format: D = 5120: 3 warps x the full 64 elements at 83 % beat 5 warps x 32 elements at
+// 100 % by 3-6 %; D = 3072 with 32-element pieces: 2 warps x 64 at 75 % beat 3 warps x 32 at 100 % by 2 %, with
+// 16-element pieces the two are level (hence the handicap of a half-filled lane: 0.26 and 0.2).
 static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
 {
     const int maxp = MXN_FWD_MAX_ELEMS / B;
@@ -634,7 +637,7 @@ static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
             const long lanes = (long)32 * w * p;
             if (!exists || lanes < K) continue;
             const int elems = p * B;   // per lane
-            const double handicap = w == 1 || elems >= MXN_FWD_MAX_ELEMS ? 0.0 : elems >= MXN_FWD_MAX_ELEMS / 2 ? 0.15 : 0.45;
+            const double handicap = w == 1 || elems >= MXN_FWD_MAX_ELEMS ? 0.0 : elems >= MXN_FWD_MAX_ELEMS / 2 ? (B == 32 ? 0.26 : 0.2) : 0.45;
             const double cost = (double)(lanes - K) / (double)lanes + handicap;
             if (best_cost < 0.0 || cost < best_cost - 1e-9) {
                 best_cost = cost;
