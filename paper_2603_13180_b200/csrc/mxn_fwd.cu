@@ -62,7 +62,7 @@ __device__ __forceinline__ void prefetch_row(const uint16_t* base, int64_t row, 
 }
 
 template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER, int LPB = 1>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, GAIN)) fwd_e4m3_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_e4m3_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, MXN_FWD_MIN_CTAS) fwd_add
 
 // plain MXCast to E5M2 codes (gradient tensors), the paper's rounding rule with 2^15
 template <int B, int NPASS, int WPR, int LPB = 1>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false)) cast_e5m2_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) cast_e5m2_kernel(const FwdParams P)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int group = warp / WPR, w = warp - group * WPR;
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false))
 
 // E2M1 codes with E8M0 scales (MXFP4): no gain, the paper's rounding rule
 template <int B, int NPASS, int WPR, int STAT, int LPB = 1>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false)) fwd_mxfp4_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_mxfp4_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false))
 }
 
 template <int NPASS, int WPR, int STAT>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false)) fwd_nvfp4_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_nvfp4_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false))
 // NVFP4 with two blocks per lane and pass (rows of an even number of blocks): see quantise_pair_nvfp4
 // (four-warp CTAs at 64 registers, 8 CTAs per SM: 26.5 -> 26.0 us at [16384,4096] against 66 registers, 7 CTAs)
 template <int NPASS, int WPR, int STAT>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false)) fwd_nvfp4_pair_kernel(const FwdParams P)
+__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_nvfp4_pair_kernel(const FwdParams P)
 {
     __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR, false))
 // D = 2560 (CH = 160, one row per warp) and D = 1280 (CH = 80, two rows per warp).  The row statistics are independent
 // shuffle reductions, one per row.
 template <int E, int LPB, int NPASS, int RPW, int CH, int STAT, int FMT>
-__global__ void __launch_bounds__(MXN_FWD_WARPS * 32, MXN_FWD_MIN_CTAS) fwd_multi_kernel(const FwdParams P)
+__global__ void __launch_bounds__(MXN_FWD_WARPS * 32, 32 / MXN_FWD_WARPS) fwd_multi_kernel(const FwdParams P)
 {
     constexpr int W = E / 2;
     static_assert(RPW * CH <= 32 * NPASS && CH % LPB == 0 && (E == 16 || E == 32), "the run fits the warp's passes; 32- or 64-byte pieces");
@@ -431,7 +431,7 @@ template <int B, int LPB, int STAT, bool GAIN, bool PAPER>
 static fwd_fn pick_e4m3(int wpr, int npass)
 {
     constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    constexpr bool FINE = !GAIN && PAPER && STAT != STAT_POSTROUND;
+    constexpr bool FINE = PAPER && STAT != STAT_POSTROUND;
     if (wpr > 1) {
         if (npass == MAXP) return e4m3_by_wpr<B, LPB, MAXP, STAT, GAIN, PAPER, FINE>(wpr);
         if (FINE && MAXP >= 4 && npass == MAXP / 2) return e4m3_by_wpr<B, LPB, (MAXP >= 4 ? MAXP / 2 : 1), STAT, GAIN, PAPER, FINE>(wpr);
@@ -446,20 +446,38 @@ static fwd_fn pick_e4m3(int wpr, int npass)
     }
 }
 template <int B, int LPB, bool PAPER>
-static fwd_fn pick_stat(int stat, bool gain, int wpr, int npass)
+static fwd_fn pick_stat(int stat, int wpr, int npass)
 {
     switch (stat) {
         case STAT_NONE: return pick_e4m3<B, LPB, STAT_NONE, false, PAPER>(wpr, npass);
-        case STAT_RMS: return gain ? pick_e4m3<B, LPB, STAT_RMS, true, PAPER>(wpr, npass) : pick_e4m3<B, LPB, STAT_RMS, false, PAPER>(wpr, npass);
-        case STAT_MX: return gain ? pick_e4m3<B, LPB, STAT_MX, true, PAPER>(wpr, npass) : pick_e4m3<B, LPB, STAT_MX, false, PAPER>(wpr, npass);
-        case STAT_POSTROUND: return (gain || !PAPER) ? nullptr : pick_e4m3<B, LPB, STAT_POSTROUND, false, true>(wpr, npass);
+        case STAT_RMS: return pick_e4m3<B, LPB, STAT_RMS, false, PAPER>(wpr, npass);
+        case STAT_MX: return pick_e4m3<B, LPB, STAT_MX, false, PAPER>(wpr, npass);
+        case STAT_POSTROUND: return !PAPER ? nullptr : pick_e4m3<B, LPB, STAT_POSTROUND, false, true>(wpr, npass);
         default: return nullptr;
     }
 }
 template <int B, int LPB>
-static fwd_fn pick_round(int round, int stat, bool gain, int wpr, int npass)
+static fwd_fn pick_round(int round, int stat, int wpr, int npass)
 {
-    return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, LPB, true>(stat, gain, wpr, npass) : pick_stat<B, LPB, false>(stat, gain, wpr, npass);
+    return round == MXN_ROUND_RCEIL_POW2 ? pick_stat<B, LPB, true>(stat, wpr, npass) : pick_stat<B, LPB, false>(stat, wpr, npass);
+}
+// With a gain a lane always holds 16-element pieces (a block of 32 or 64 is shared by 2 or 4 lanes): the products
+// x * rho * gamma of a piece stay in registers between the block maximum and the conversion, and 16 of them fit the
+// 64 registers that 32 resident warps per SM allow, 32 do not (measured at [16384, 4096], block 32: 37.3 us as 32-element
+// pieces, 32.2 us as 16-element pieces; 42.7 us before, with scalar arithmetic and no register limit).
+template <int LPB, bool PAPER>
+static fwd_fn pick_gain_stat(int stat, int wpr, int npass)
+{
+    switch (stat) {
+        case STAT_RMS: return pick_e4m3<16, LPB, STAT_RMS, true, PAPER>(wpr, npass);
+        case STAT_MX: return pick_e4m3<16, LPB, STAT_MX, true, PAPER>(wpr, npass);
+        default: return nullptr;
+    }
+}
+template <int LPB>
+static fwd_fn pick_gain_round(int round, int stat, int wpr, int npass)
+{
+    return round == MXN_ROUND_RCEIL_POW2 ? pick_gain_stat<LPB, true>(stat, wpr, npass) : pick_gain_stat<LPB, false>(stat, wpr, npass);
 }
 template <int B, int LPB, int NPASS, int STAT>
 static fwd_fn mxfp4_by_wpr(int wpr)
@@ -621,7 +639,8 @@ static fwd_fn pick_nvfp4_pair(int wpr, int npass)
 // D = 2560, B = 16: 5 warps x 1 pass (16 elements per lane) at 100 % lost to 2 warps x 4 passes at 62.5 %.
 // Measured at 32768 rows, every format: D = 5120: 3 warps x the full 64 elements at 83 % beat 5 warps x 32 elements at
 // 100 % by 3-6 %; D = 3072 with 32-element pieces: 2 warps x 64 at 75 % beat 3 warps x 32 at 100 % by 2 %, with
-// 16-element pieces the two are level (hence the handicap of a half-filled lane: 0.26 and 0.2).
+// 16-element pieces the two are level; D = 2560 with 16-element pieces and a gain: 2 warps x 64 at 62.5 % beat 3 warps x 32
+// at 83 % (26.3 against 28.2 us at 16384 rows).  Hence the handicap of a half-filled lane: 0.26 and 0.22.
 static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
 {
     const int maxp = MXN_FWD_MAX_ELEMS / B;
@@ -637,7 +656,7 @@ static bool plan_row(int K, int B, bool fine, bool nvfp4, int* wpr, int* npass)
             const long lanes = (long)32 * w * p;
             if (!exists || lanes < K) continue;
             const int elems = p * B;   // per lane
-            const double handicap = w == 1 || elems >= MXN_FWD_MAX_ELEMS ? 0.0 : elems >= MXN_FWD_MAX_ELEMS / 2 ? (B == 32 ? 0.26 : 0.2) : 0.45;
+            const double handicap = w == 1 || elems >= MXN_FWD_MAX_ELEMS ? 0.0 : elems >= MXN_FWD_MAX_ELEMS / 2 ? (B == 32 ? 0.26 : 0.22) : 0.45;
             const double cost = (double)(lanes - K) / (double)lanes + handicap;
             if (best_cost < 0.0 || cost < best_cost - 1e-9) {
                 best_cost = cost;
@@ -674,9 +693,10 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     // 1-3 % faster than one block per lane up to D = 10240 and 2-10 % slower from D = 12288 on (65536 rows), hence the limit.
     const bool nv_pair = nvfp4 && P.K % 2 == 0 && P.D < 12288;
 #endif
-    const int E = nv_pair ? 32 : B == 64 ? 32 : B;   // elements per lane and pass; a block of 64 is shared by two lanes
-    const bool fine = nvfp4 || mxfp4 || (!e5m2 && !add && stat != STAT_POSTROUND && P.gain == nullptr &&
-                                P.round == MXN_ROUND_RCEIL_POW2);
+    const bool has_gain = P.gain != nullptr && P.elem == ELEM_E4M3 && !add;
+    // elements per lane and pass; a block of 64 is shared by two lanes, with a gain every block by lanes of 16 elements
+    const int E = nv_pair ? 32 : has_gain ? 16 : B == 64 ? 32 : B;
+    const bool fine = nvfp4 || mxfp4 || (!e5m2 && !add && stat != STAT_POSTROUND && P.round == MXN_ROUND_RCEIL_POW2);
     P.pr_table = B == 16 ? 0 : B == 32 ? 1 : 2;
     P.chunks = nv_pair ? P.K / 2 : P.K * (B / E);
     if (!plan_row(P.chunks, E, fine, nvfp4 && !nv_pair, &P.wpr, &P.npass)) return false;
@@ -687,9 +707,8 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     }
     const int warps = cta_warps(P.wpr);
     P.rows_per_cta = rows_per_cta(P.wpr);
-    const bool has_gain = P.gain != nullptr;
     fwd_fn fn = nullptr;
-    if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && (fine || mxfp4) && stat != STAT_POSTROUND) {
+    if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && !has_gain && (fine || mxfp4) && stat != STAT_POSTROUND) {
         fn = nvfp4 ? pick_multi_stat<2>(16, stat, rpw) : mxfp4 ? pick_multi_stat<1>(B, stat, rpw) : pick_multi_stat<0>(B, stat, rpw);
         *fn_out = fn;
         *ctas_out = (P.T + (int64_t)MXN_FWD_WARPS * rpw - 1) / ((int64_t)MXN_FWD_WARPS * rpw);
@@ -702,9 +721,11 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     else if (e5m2) fn = B == 16 ? pick_e5m2<16, 1>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32, 1>(P.wpr, P.npass) : pick_e5m2<32, 2>(P.wpr, P.npass);
     else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16, 1>(stat, P.wpr, P.npass)
                        : B == 32 ? pick_mxfp4_stat<32, 1>(stat, P.wpr, P.npass) : pick_mxfp4_stat<32, 2>(stat, P.wpr, P.npass);
-    else if (B == 16) fn = pick_round<16, 1>(P.round, stat, has_gain, P.wpr, P.npass);
-    else if (B == 32) fn = pick_round<32, 1>(P.round, stat, has_gain, P.wpr, P.npass);
-    else fn = pick_round<32, 2>(P.round, stat, has_gain, P.wpr, P.npass);
+    else if (has_gain) fn = B == 16 ? pick_gain_round<1>(P.round, stat, P.wpr, P.npass)
+                          : B == 32 ? pick_gain_round<2>(P.round, stat, P.wpr, P.npass) : pick_gain_round<4>(P.round, stat, P.wpr, P.npass);
+    else if (B == 16) fn = pick_round<16, 1>(P.round, stat, P.wpr, P.npass);
+    else if (B == 32) fn = pick_round<32, 1>(P.round, stat, P.wpr, P.npass);
+    else fn = pick_round<32, 2>(P.round, stat, P.wpr, P.npass);
     *fn_out = fn;
     *ctas_out = (P.T + P.rows_per_cta - 1) / P.rows_per_cta;
     *threads_out = warps * kWarp;

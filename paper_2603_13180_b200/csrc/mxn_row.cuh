@@ -23,9 +23,10 @@ namespace mxn {
 // warps of a CTA whose rows each span WPR warps
 __host__ __device__ constexpr int rows_per_cta(int wpr) { return MXN_FWD_WARPS / wpr > 1 ? MXN_FWD_WARPS / wpr : 1; }
 __host__ __device__ constexpr int cta_warps(int wpr) { return wpr * rows_per_cta(wpr); }
-// occupancy hint: the four-warp CTAs of the kernels without gain fit 64 registers per thread, i.e. 8 CTAs per SM
-// (one register more costs a whole CTA per SM: 7 instead of 8)
-__host__ __device__ constexpr int fwd_min_ctas(int wpr, bool gain) { return (cta_warps(wpr) == 4 && !gain) ? 8 : MXN_FWD_MIN_CTAS; }
+// occupancy hint: the kernels are held to 64 registers per thread, i.e. 32 warps per SM whatever the CTA
+// size (one register more is allocated as 72: a four-warp CTA then fits 7 times instead of 8, an eight-warp CTA 3 times
+// instead of 4, a sixteen-warp CTA once instead of twice)
+__host__ __device__ constexpr int fwd_min_ctas(int wpr) { return 32 / cta_warps(wpr); }
 
 // ---- post-round estimator tables (appendix "Post-round MXNorm") ------------------------------------
 // f^-1 sampled at the 65 nodes 2^(i/64) of [1,2] for each block size, with the slope of every interval;
@@ -314,24 +315,28 @@ __device__ __forceinline__ void quantise_store_e4m3(const uint32_t (&xr)[NPASS][
 #pragma unroll
                 for (int j = 0; j < W; ++j) gr[j] = 0u;
             }
-            float my = 0.0f;
+            // two elements per instruction (packed binary32 multiplies, each half an ordinary IEEE operation)
+            const float2 rr = make_float2(rho, rho);
+            // the block's products are kept between the maximum and the conversion (the lane's input words of this
+            // block and the gain are dead by then)
+            float2 y[W];
+            float2 my2 = make_float2(0.0f, 0.0f);
 #pragma unroll
             for (int j = 0; j < W; ++j) {
-                const float y0 = __fmul_rn(__fmul_rn(bf16_lo(xr[i][j]), rho), bf16_lo(gr[j]));
-                const float y1 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), bf16_hi(gr[j]));
-                my = fmaxf(my, fmaxf(fabsf(y0), fabsf(y1)));
+                y[j] = mul2(mul2(bf16x2_to_f32x2(xr[i][j]), rr), bf16x2_to_f32x2(gr[j]));
+                my2.x = fmaxf(my2.x, fabsf(y[j].x));
+                my2.y = fmaxf(my2.y, fabsf(y[j].y));
             }
+            float my = fmaxf(my2.x, my2.y);
 #pragma unroll
             for (int o = 1; o < LPB; o <<= 1) my = fmaxf(my, __shfl_xor_sync(0xFFFFFFFFu, my, o));
             sb = PAPER ? e8m0_scale_rceil_pow2<ELEM == 2 ? 15 : 8>(my) : e8m0_scale(my, P.round);
             const float inv = inv_scale(sb);
+            const float2 ii = make_float2(inv, inv);
 #pragma unroll
             for (int j = 0; j < W; j += 2) {
-                const float y0 = __fmul_rn(__fmul_rn(bf16_lo(xr[i][j]), rho), bf16_lo(gr[j]));
-                const float y1 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j]), rho), bf16_hi(gr[j]));
-                const float y2 = __fmul_rn(__fmul_rn(bf16_lo(xr[i][j + 1]), rho), bf16_lo(gr[j + 1]));
-                const float y3 = __fmul_rn(__fmul_rn(bf16_hi(xr[i][j + 1]), rho), bf16_hi(gr[j + 1]));
-                out[j / 2] = cvt_fp8x4<ELEM>(__fmul_rn(y0, inv), __fmul_rn(y1, inv), __fmul_rn(y2, inv), __fmul_rn(y3, inv));
+                const float2 qa = mul2(y[j], ii), qb = mul2(y[j + 1], ii);
+                out[j / 2] = cvt_fp8x4<ELEM>(qa.x, qa.y, qb.x, qb.y);
             }
         }
         if (active) {

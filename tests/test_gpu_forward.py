@@ -63,7 +63,9 @@ def test_rmsnorm_mxfp8_fwd_matches_oracle(binding, oracle, T, D):
 
 @pytest.mark.parametrize("block", [16, 64])
 @pytest.mark.parametrize("T,D", [(3, 64), (19, 1024), (5, 2048), (9, 2560), (130, 2560), (6, 3072), (7, 4096), (4, 8192), (3, 16384),
-                                 (10, 1536), (6, 3584), (11, 1280), (133, 1280)])
+                                 (10, 1536), (6, 3584), (11, 1280), (133, 1280),
+                                 # with a gain every block size runs as 16-element pieces: rows of 3, 5, 6, 7 and 16 warps
+                                 (3, 5120), (5, 6144), (3, 7168), (2, 10240), (2, 12288), (2, 14336), (2, 32768)])
 def test_other_block_sizes(binding, oracle, T, D, block):
     x, gain = rows(T, D, seed=T + D + block)
     got = gu.run_fwd(binding, oracle, "mx", x, block=block, eps=1e-5)
@@ -79,9 +81,10 @@ def test_other_block_sizes(binding, oracle, T, D, block):
         gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, block=block, eps=1e-5), f"mxnorm with gain B={block} layout={layout}")
 
 
+@pytest.mark.parametrize("T,D", [(41, 2048), (5, 5120), (3, 12288)])
 @pytest.mark.parametrize("rnd", [1, 2])
-def test_other_rounding_modes(binding, oracle, rnd):
-    x, gain = rows(41, 2048, seed=17)
+def test_other_rounding_modes(binding, oracle, rnd, T, D):
+    x, gain = rows(T, D, seed=17 + D)
     got = gu.run_fwd(binding, oracle, "mx", x, round=rnd, eps=1e-5)
     gu.assert_exact(got, gu.run_ref(oracle, "mx", x, round=rnd, eps=1e-5), f"mxnorm round={rnd}")
     got = gu.run_fwd(binding, oracle, "mx", x, gain, round=rnd)
