@@ -490,6 +490,25 @@ def main():
 
             mspr = time_median(postround, SETS, args.steps, args.warmup, stream)
             others["mxnorm_postround_fwd"] = {"ms": mspr, "gbs": algorithmic_bytes("mx", T, D) / mspr / 1e6}
+            # the same two kernels with a gain vector (the extension of Algorithm 2; Algorithm 1 as commonly deployed)
+            gain_vec = (1.0 + 0.1 * torch.randn(D, device="cuda")).to(torch.bfloat16)
+
+            def fwd_gain(i):
+                c, s, r = outs[i]
+                st = L.mxnorm_fwd(xs[i].data_ptr(), gain_vec.data_ptr(), T, D, 32, 2, 0.0, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(), 0, layout, sh)
+                if st != 0:
+                    raise RuntimeError(mx.status_string(st))
+
+            def rms_gain(i):
+                c, s, r = outs[i]
+                st = L.rmsnorm_mxfp8_fwd(xs[i].data_ptr(), gain_vec.data_ptr(), T, D, 32, EPS, c.data_ptr(), s.data_ptr(), r.data_ptr(), 0, layout, sh)
+                if st != 0:
+                    raise RuntimeError(mx.status_string(st))
+
+            msg = time_median(fwd_gain, SETS, args.steps, args.warmup, stream)
+            others["mxnorm_fwd_with_gain"] = {"ms": msg, "gbs": (algorithmic_bytes("mx", T, D) + 2 * D) / msg / 1e6}
+            msg = time_median(rms_gain, SETS, args.steps, args.warmup, stream)
+            others["rmsnorm_mxfp8_fwd_with_gain"] = {"ms": msg, "gbs": (algorithmic_bytes("rms", T, D) + 2 * D) / msg / 1e6}
             hs = [torch.empty_like(xs[0]) for _ in range(SETS)]
 
             def add_fwd(i):
