@@ -709,7 +709,8 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     const int warps = cta_warps(P.wpr);
     P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
-    if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && !has_gain && (fine || mxfp4) && stat != STAT_POSTROUND) {
+    // (the one-warp kernel has the paper's rounding rule compiled in and takes no gain)
+    if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && !has_gain && (nvfp4 || mxfp4 || P.round == MXN_ROUND_RCEIL_POW2) && (fine || mxfp4) && stat != STAT_POSTROUND) {
         fn = nvfp4 ? pick_multi_stat<2>(16, stat, rpw) : mxfp4 ? pick_multi_stat<1>(B, stat, rpw) : pick_multi_stat<0>(B, stat, rpw);
         *fn_out = fn;
         *ctas_out = (P.T + (int64_t)MXN_FWD_WARPS * rpw - 1) / ((int64_t)MXN_FWD_WARPS * rpw);

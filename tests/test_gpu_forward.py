@@ -81,7 +81,7 @@ def test_other_block_sizes(binding, oracle, T, D, block):
         gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, block=block, eps=1e-5), f"mxnorm with gain B={block} layout={layout}")
 
 
-@pytest.mark.parametrize("T,D", [(41, 2048), (5, 5120), (3, 12288)])
+@pytest.mark.parametrize("T,D", [(41, 2048), (9, 2560), (5, 5120), (3, 12288)])
 @pytest.mark.parametrize("rnd", [1, 2])
 def test_other_rounding_modes(binding, oracle, rnd, T, D):
     x, gain = rows(T, D, seed=17 + D)
