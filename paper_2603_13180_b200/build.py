@@ -8,8 +8,8 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmxnorm.so")
-SOURCES = ["mxn_api.cu", "mxn_fwd.cu", "mxn_bwd.cu", "mxn_transposed.cu"]
-HEADERS = ["mxn_device.cuh", "mxn_internal.h", "mxn_row.cuh", "mxn_col.cuh", os.path.join("..", "..", "include", "mxnorm.h")]
+SOURCES = ["mxn_api.cu", "mxn_fwd.cu", "mxn_fwd_fp4.cu", "mxn_bwd.cu", "mxn_transposed.cu"]
+HEADERS = ["mxn_device.cuh", "mxn_internal.h", "mxn_row.cuh", "mxn_fwd_common.cuh", "mxn_col.cuh", os.path.join("..", "..", "include", "mxnorm.h")]
 
 # No fast-math and no flush-to-zero: scale selection relies on IEEE division, subnormals and exact
 # power-of-two products.

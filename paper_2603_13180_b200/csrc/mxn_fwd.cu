@@ -25,41 +25,9 @@
 #include "mxn_device.cuh"
 #include "mxn_internal.h"
 #include "mxn_row.cuh"
+#include "mxn_fwd_common.cuh"
 
 namespace mxn {
-
-// ---- register-direct kernels: one row per row group, loaded straight from global memory -----------
-// Generic path: any D % B == 0, rows spanning up to 8 warps, optional gain.
-template <int B, int NPASS, bool COHERENT = false>
-__device__ __forceinline__ void load_row_direct(uint32_t (&xr)[NPASS][B / 2], const uint16_t* xrow, int K, int wpr, int w, int lane)
-{
-    constexpr int W = B / 2;
-#pragma unroll
-    for (int i = 0; i < NPASS; ++i) {
-        const int k = (i * wpr + w) * kWarp + lane;
-        if (k < K) {
-            const uint16_t* p = xrow + (int64_t)k * B;
-#pragma unroll
-            for (int v = 0; v < W / 8; ++v) {
-                if (COHERENT) ld_v8_coherent(p + v * 16, &xr[i][v * 8]);
-                else ld_v8(p + v * 16, &xr[i][v * 8]);
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < W; ++j) xr[i][j] = 0u;
-        }
-    }
-}
-
-constexpr unsigned kFirstWaveCtas = 148 * 8;   // SMs x the most CTAs of 128 threads an SM holds at 64 registers
-
-// One lane per row asks for the whole row in L2 before the kernel waits for its predecessor (see prefetch_l2_bulk):
-// rows are multiples of 32 bytes and 32-byte aligned.
-__device__ __forceinline__ void prefetch_row(const uint16_t* base, int64_t row, const FwdParams& P, int w, int lane)
-{
-    // only CTAs of the first wave can be resident before the previous kernel has ended; for the rest the hint is redundant
-    if (w == 0 && lane == 0 && row < P.T && blockIdx.x < kFirstWaveCtas) prefetch_l2_bulk(base + row * P.D, (uint32_t)P.D * 2u);
-}
 
 template <int B, int NPASS, int WPR, int STAT, bool GAIN, bool PAPER, int LPB = 1>
 __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_e4m3_kernel(const FwdParams P)
@@ -151,111 +119,6 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) cast_e
     load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
     (void)block_stats<B, NPASS, STAT_NONE, LPB>(xr, m, 2, lane);
     quantise_store_e4m3<B, NPASS, WPR, false, true, 2, LPB>(xr, m, 1.0f, P, row, w, lane);
-}
-
-// E2M1 codes with E8M0 scales (MXFP4): no gain, the paper's rounding rule
-template <int B, int NPASS, int WPR, int STAT, int LPB = 1>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_mxfp4_kernel(const FwdParams P)
-{
-    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int group = warp / WPR, w = warp - group * WPR;
-    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
-    prefetch_row(P.x, row, P, w, lane);
-    pdl_prologue();
-    if (row >= P.T) return;
-
-    uint32_t xr[NPASS][B / 2];
-    float m[NPASS];
-    load_row_direct<B, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
-    double stat = block_stats<B, NPASS, STAT, LPB>(xr, m, P.p, lane);
-    if (STAT == STAT_RMS) forget_unpacked<NPASS, B / 2>(xr);
-    float r = 1.0f, rho = 1.0f;
-    if (STAT != STAT_NONE) {
-        stat = group_sum<WPR>(stat, group, w, red);
-        finish_stat<STAT>(stat, P, r, rho);
-        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
-    }
-    quantise_store_mxfp4<B, NPASS, WPR, LPB>(xr, m, rho, P, row, w, lane);
-}
-
-template <int NPASS, int WPR, int STAT>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_nvfp4_kernel(const FwdParams P)
-{
-    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int group = warp / WPR, w = warp - group * WPR;
-    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
-    prefetch_row(P.x, row, P, w, lane);
-    pdl_prologue();
-    if (row >= P.T) return;
-
-    uint32_t xr[NPASS][8];
-    float m[NPASS];
-    load_row_direct<16, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
-    double stat = block_stats<16, NPASS, STAT>(xr, m, P.p);
-    if (STAT == STAT_RMS) forget_unpacked<NPASS, 8>(xr);
-    float r = 1.0f, rho = 1.0f;
-    if (STAT != STAT_NONE) {
-        stat = group_sum<WPR>(stat, group, w, red);
-        finish_stat<STAT>(stat, P, r, rho);
-        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
-    }
-    quantise_store_nvfp4<NPASS, WPR>(xr, m, rho, P, row, w, lane);
-}
-
-// NVFP4 with two blocks per lane and pass (rows of an even number of blocks): see quantise_pair_nvfp4
-// (four-warp CTAs at 64 registers, 8 CTAs per SM: 26.5 -> 26.0 us at [16384,4096] against 66 registers, 7 CTAs)
-template <int NPASS, int WPR, int STAT>
-__global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) fwd_nvfp4_pair_kernel(const FwdParams P)
-{
-    __shared__ double red[WPR > 1 ? cta_warps(WPR) : 1];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int group = warp / WPR, w = warp - group * WPR;
-    const int64_t row = (int64_t)blockIdx.x * rows_per_cta(WPR) + group;
-    prefetch_row(P.x, row, P, w, lane);
-    pdl_prologue();
-    if (row >= P.T) return;
-
-    uint32_t xr[NPASS][16];
-    float m0[NPASS], m1[NPASS];
-    load_row_direct<32, NPASS>(xr, P.x + row * P.D, P.chunks, WPR, w, lane);
-    double stat = 0.0;
-    float2 ssa = make_float2(0.f, 0.f), ssb = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int i = 0; i < NPASS; ++i) {
-        uint32_t ma = absmax_bf16x2(xr[i][0], xr[i][1]), mb = absmax_bf16x2(xr[i][8], xr[i][9]);
-#pragma unroll
-        for (int j = 2; j < 8; ++j) {
-            ma = absmax_bf16x2(ma, xr[i][j]);
-            mb = absmax_bf16x2(mb, xr[i][8 + j]);
-        }
-        m0[i] = hmax_abs_to_f32(ma);
-        m1[i] = hmax_abs_to_f32(mb);
-        if (STAT == STAT_MX) {
-            const double d0 = (double)m0[i], d1 = (double)m1[i];
-            stat = P.p == 2 ? __fma_rn(d1, d1, __fma_rn(d0, d0, stat)) : __dadd_rn(__dadd_rn(stat, d0), d1);
-        }
-        if (STAT == STAT_RMS) {
-#pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-                const float2 a = bf16x2_to_f32x2(xr[i][j]), b = bf16x2_to_f32x2(xr[i][j + 1]);
-                ssa = __ffma2_rn(a, a, ssa);
-                ssb = __ffma2_rn(b, b, ssb);
-            }
-        }
-    }
-    if (STAT == STAT_RMS) {
-        stat = (double)ssa.x + (double)ssa.y + ((double)ssb.x + (double)ssb.y);
-        forget_unpacked<NPASS, 16>(xr);
-    }
-    float r = 1.0f, rho = 1.0f;
-    if (STAT != STAT_NONE) {
-        stat = group_sum<WPR>(stat, group, w, red);
-        finish_stat<STAT>(stat, P, r, rho);
-        if (P.rms_out != nullptr && w == 0 && lane == 0) P.rms_out[row] = r;
-    }
-    quantise_store_nvfp4_pair<NPASS, WPR>(xr, m0, m1, rho, P, row, w, lane);
 }
 
 // ---- one warp per run of RPW short rows ------------------------------------------------------------------------------
@@ -392,7 +255,6 @@ __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, 32 / MXN_FWD_WARPS) fwd_mu
 }
 
 // ---- dispatch ---------------------------------------------------------------------------------
-typedef void (*fwd_fn)(const FwdParams);
 
 // In the templates below B is the number of elements a lane holds per pass and LPB the lanes per block
 // (block size of the format = B * LPB: 16 = 16x1, 32 = 32x1, 64 = 32x2).
@@ -480,41 +342,6 @@ static fwd_fn pick_gain_round(int round, int stat, int wpr, int npass)
 {
     return round == MXN_ROUND_RCEIL_POW2 ? pick_gain_stat<LPB, true>(stat, wpr, npass) : pick_gain_stat<LPB, false>(stat, wpr, npass);
 }
-template <int B, int LPB, int NPASS, int STAT>
-static fwd_fn mxfp4_by_wpr(int wpr)
-{
-    switch (wpr) {
-        case 1: return fwd_mxfp4_kernel<B, NPASS, 1, STAT, LPB>;
-        case 2: return fwd_mxfp4_kernel<B, NPASS, 2, STAT, LPB>;
-        case 3: return fwd_mxfp4_kernel<B, NPASS, 3, STAT, LPB>;
-        case 4: return fwd_mxfp4_kernel<B, NPASS, 4, STAT, LPB>;
-        case 5: return fwd_mxfp4_kernel<B, NPASS, 5, STAT, LPB>;
-        case 6: return fwd_mxfp4_kernel<B, NPASS, 6, STAT, LPB>;
-        case 7: return fwd_mxfp4_kernel<B, NPASS, 7, STAT, LPB>;
-        case 8: return fwd_mxfp4_kernel<B, NPASS, 8, STAT, LPB>;
-        case 16: return fwd_mxfp4_kernel<B, NPASS, 16, STAT, LPB>;
-        default: return nullptr;
-    }
-}
-// the same set of (warps per row, passes) as the E4M3 headline kernels: every count in kFineWpr with the full pass
-// count, half of it (four-pass kernels) or one pass; one warp per row with any pass count
-template <int B, int LPB, int STAT>
-static fwd_fn pick_mxfp4(int wpr, int npass)
-{
-    constexpr int MAXP = MXN_FWD_MAX_ELEMS / B;
-    if (wpr > 1) {
-        if (npass == MAXP) return mxfp4_by_wpr<B, LPB, MAXP, STAT>(wpr);
-        if (MAXP >= 4 && npass == MAXP / 2) return mxfp4_by_wpr<B, LPB, (MAXP >= 4 ? MAXP / 2 : 1), STAT>(wpr);
-        if (npass == 1) return mxfp4_by_wpr<B, LPB, 1, STAT>(wpr);
-        return nullptr;
-    }
-    switch (npass) {
-        case 1: return fwd_mxfp4_kernel<B, 1, 1, STAT, LPB>;
-        case 2: return fwd_mxfp4_kernel<B, (MAXP >= 2 ? 2 : MAXP), 1, STAT, LPB>;
-        case 3: return fwd_mxfp4_kernel<B, (MAXP >= 3 ? 3 : MAXP), 1, STAT, LPB>;
-        default: return fwd_mxfp4_kernel<B, MAXP, 1, STAT, LPB>;
-    }
-}
 template <int B, int LPB>
 static fwd_fn pick_add_mx(int wpr, int npass)
 {
@@ -549,39 +376,7 @@ static fwd_fn pick_e5m2(int wpr, int npass)
     }
 }
 
-template <int B, int LPB>
-static fwd_fn pick_mxfp4_stat(int stat, int wpr, int npass)
-{
-    if (stat == STAT_MX) return pick_mxfp4<B, LPB, STAT_MX>(wpr, npass);
-    if (stat == STAT_RMS) return pick_mxfp4<B, LPB, STAT_RMS>(wpr, npass);
-    return pick_mxfp4<B, LPB, STAT_NONE>(wpr, npass);
-}
 
-template <int NPASS, int STAT>
-static fwd_fn nvfp4_by_wpr(int wpr)
-{
-    switch (wpr) {
-        case 1: return fwd_nvfp4_kernel<NPASS, 1, STAT>;
-        case 2: return fwd_nvfp4_kernel<NPASS, 2, STAT>;
-        case 3: return fwd_nvfp4_kernel<NPASS, 3, STAT>;
-        case 4: return fwd_nvfp4_kernel<NPASS, 4, STAT>;
-        case 5: return fwd_nvfp4_kernel<NPASS, 5, STAT>;
-        case 6: return fwd_nvfp4_kernel<NPASS, 6, STAT>;
-        case 7: return fwd_nvfp4_kernel<NPASS, 7, STAT>;
-        case 8: return fwd_nvfp4_kernel<NPASS, 8, STAT>;
-        case 16: return fwd_nvfp4_kernel<NPASS, 16, STAT>;
-        default: return nullptr;
-    }
-}
-template <int STAT>
-static fwd_fn pick_nvfp4(int wpr, int npass)
-{
-    constexpr int MAXP = MXN_FWD_MAX_ELEMS / 16;
-    if (npass == MAXP) return nvfp4_by_wpr<MAXP, STAT>(wpr);
-    if (npass == MAXP / 2) return nvfp4_by_wpr<(MAXP >= 2 ? MAXP / 2 : 1), STAT>(wpr);
-    if (npass == 1) return nvfp4_by_wpr<1, STAT>(wpr);
-    return nullptr;
-}
 
 // The one-warp kernel with 16-element pieces is used where it measured faster than the row-group kernels: rows of
 // 160 pieces (D = 2560: five passes of one warp instead of three warps x one pass or two warps x four passes;
@@ -611,27 +406,6 @@ static fwd_fn pick_multi_stat(int B, int stat, int rpw)
     return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B, rpw) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B, rpw) : pick_multi<FMT, STAT_NONE>(B, rpw);
 }
 
-template <int NPASS, int STAT>
-static fwd_fn nvfp4_pair_by_wpr(int wpr)
-{
-    switch (wpr) {
-        case 1: return fwd_nvfp4_pair_kernel<NPASS, 1, STAT>;
-        case 2: return fwd_nvfp4_pair_kernel<NPASS, 2, STAT>;
-        case 3: return fwd_nvfp4_pair_kernel<NPASS, 3, STAT>;
-        case 4: return fwd_nvfp4_pair_kernel<NPASS, 4, STAT>;
-        case 5: return fwd_nvfp4_pair_kernel<NPASS, 5, STAT>;
-        case 6: return fwd_nvfp4_pair_kernel<NPASS, 6, STAT>;
-        case 7: return fwd_nvfp4_pair_kernel<NPASS, 7, STAT>;
-        case 8: return fwd_nvfp4_pair_kernel<NPASS, 8, STAT>;
-        case 16: return fwd_nvfp4_pair_kernel<NPASS, 16, STAT>;
-        default: return nullptr;
-    }
-}
-template <int STAT>
-static fwd_fn pick_nvfp4_pair(int wpr, int npass)
-{
-    return npass == 2 ? nvfp4_pair_by_wpr<2, STAT>(wpr) : npass == 1 ? nvfp4_pair_by_wpr<1, STAT>(wpr) : nullptr;
-}
 
 // Splits the K per-lane pieces of a row (B elements each) over WPR warps x NPASS passes (at most MXN_FWD_MAX_ELEMS
 // elements per lane), choosing among the instantiated kernels by the fraction of idle lanes, with a handicap for
@@ -691,7 +465,7 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     const bool nv_pair = false;
 #else
     // NVFP4 rows of an even number of blocks: a lane owns two adjacent blocks (about a fifth fewer instructions).  Measured
-    // 1-3 % faster than one block per lane up to D = 10240 and 2-10 % slower from D = 12288 on (65536 rows), hence the limit.
+    // 0-2 % faster than one block per lane up to D = 12288, level at 14336 and 1 % slower at 16384, hence the limit.
     const bool nv_pair = nvfp4 && P.K % 2 == 0 && P.D < 12288;
 #endif
     const bool has_gain = P.gain != nullptr && P.elem == ELEM_E4M3 && !add;
@@ -717,12 +491,9 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
         *threads_out = MXN_FWD_WARPS * kWarp;
         return fn != nullptr;
     }
-    if (nv_pair) fn = stat == STAT_RMS ? pick_nvfp4_pair<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4_pair<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4_pair<STAT_MX>(P.wpr, P.npass);
-    else if (nvfp4) fn = stat == STAT_RMS ? pick_nvfp4<STAT_RMS>(P.wpr, P.npass) : stat == STAT_NONE ? pick_nvfp4<STAT_NONE>(P.wpr, P.npass) : pick_nvfp4<STAT_MX>(P.wpr, P.npass);
+    if (nvfp4 || mxfp4) fn = pick_fp4_kernel(nvfp4, nv_pair, B, stat, P.wpr, P.npass);
     else if (add) fn = B == 16 ? pick_add_mx<16, 1>(P.wpr, P.npass) : B == 32 ? pick_add_mx<32, 1>(P.wpr, P.npass) : pick_add_mx<32, 2>(P.wpr, P.npass);
     else if (e5m2) fn = B == 16 ? pick_e5m2<16, 1>(P.wpr, P.npass) : B == 32 ? pick_e5m2<32, 1>(P.wpr, P.npass) : pick_e5m2<32, 2>(P.wpr, P.npass);
-    else if (mxfp4) fn = B == 16 ? pick_mxfp4_stat<16, 1>(stat, P.wpr, P.npass)
-                       : B == 32 ? pick_mxfp4_stat<32, 1>(stat, P.wpr, P.npass) : pick_mxfp4_stat<32, 2>(stat, P.wpr, P.npass);
     else if (has_gain) fn = B == 16 ? pick_gain_round<1>(P.round, stat, P.wpr, P.npass)
                           : B == 32 ? pick_gain_round<2>(P.round, stat, P.wpr, P.npass) : pick_gain_round<4>(P.round, stat, P.wpr, P.npass);
     else if (B == 16) fn = pick_round<16, 1>(P.round, stat, P.wpr, P.npass);
