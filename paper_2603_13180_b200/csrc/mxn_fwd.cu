@@ -125,8 +125,9 @@ __global__ void __launch_bounds__(cta_warps(WPR) * 32, fwd_min_ctas(WPR)) cast_e
 // One warp, no shared memory.  The warp takes RPW consecutive rows of CH pieces each (E = 16 elements per piece, LPB lanes
 // per block) as one contiguous run of RPW * CH pieces: piece j of the run goes to pass j / 32, lane j % 32, so every lane
 // of every pass is busy when RPW * CH = 32 NPASS, however the rows fall on the passes (CH is a compile-time constant:
-// the row of a piece is a constant division).  Used for rows of 5 * 2^r blocks that no warps-per-row split fills:
-// D = 2560 (CH = 160, one row per warp) and D = 1280 (CH = 80, two rows per warp).  The row statistics are independent
+// the row of a piece is a constant division).  Used for rows that no warps-per-row split fills (D = 2560: CH = 160, one
+// row per warp; D = 1280: CH = 80, two rows per warp; D = 1536: three passes) and for rows too short to keep a warp's
+// loads in flight (D = 512: four rows per warp; D = 768: two); see one_warp_shape.  The row statistics are independent
 // shuffle reductions, one per row.
 template <int E, int LPB, int NPASS, int RPW, int CH, int STAT, int FMT>
 __global__ void __launch_bounds__(MXN_FWD_WARPS * 32, 32 / MXN_FWD_WARPS) fwd_multi_kernel(const FwdParams P)
@@ -378,32 +379,55 @@ static fwd_fn pick_e5m2(int wpr, int npass)
 
 
 
-// The one-warp kernel with 16-element pieces is used where it measured faster than the row-group kernels: rows of
-// 160 pieces (D = 2560: five passes of one warp instead of three warps x one pass or two warps x four passes;
-// [16384, 2560]: 5.7 -> 5.9 TB/s for blocks of 32, 5.3 -> 6.1 for blocks of 16, NVFP4 4.5 -> 5.1) and rows of 80 pieces
-// (D = 1280: two rows per warp; NVFP4 only: 4.2 -> 4.5 TB/s at 16384 rows, 4.9 -> 5.5 at 65536, while the E8M0-scaled
-// formats lose 1-5 % there).  Measured and not kept: two rows of 32 pieces per warp (D = 1024: 5.5 -> 5.2 TB/s),
-// three passes of 16-element pieces (D = 1536: 5.8 -> 5.5), 8-element pieces with four lanes per block (D = 1280:
-// 5.1 -> 3.8, D = 1792: 6.1 -> 4.0), and CTA tiles of whole rows packed across warps through shared memory (two
-// CTA-wide barriers per tile: slower than one row per row group at every size but D = 2560).
-static int one_warp_rows(int64_t D, bool nvfp4) { return D == 2560 ? 1 : (D == 1280 && nvfp4) ? 2 : 0; }
+// The one-warp kernel with 16-element pieces is used where it measured faster than the row-group kernels (all variants
+// at 64 registers; [16384, D] and [65536, D]):
+//   D = 2560 (160 pieces, one row per warp: five passes of one warp instead of three warps x one pass or two warps x four
+//     passes): every format, 8-16 % faster;
+//   D = 512 (32 pieces, four rows per warp): every format and statistic, 8-58 % faster at 65536 rows, -8 ... +18 % at 16384;
+//   D = 768 (48 pieces, two rows per warp): blocks of 16 only (1-19 % faster; blocks of 32 and 64 are level);
+//   D = 1280 (80 pieces, two rows per warp): blocks of 16 with the MXNorm statistic (4-11 % faster; the sum of squares
+//     loses 2-9 % there, blocks of 32 / 64 gain 4 % at 65536 rows and lose 4 % at 16384), and NVFP4 (level);
+//   D = 1536 (96 pieces, one row per warp, three passes): NVFP4 only (6-9 % faster; the E8M0-scaled formats are level).
+// Measured and not kept: two rows of 64 pieces per warp (D = 1024: -9 ... +6 %), 8-element pieces with four lanes per
+// block (D = 1280: 5.1 -> 3.8 TB/s, D = 1792: 6.1 -> 4.0), and CTA tiles of whole rows packed across warps through shared
+// memory (two CTA-wide barriers per tile: slower than one row per row group at every size but D = 2560).
+struct MultiShape { int rpw, ch; };   // rows per warp, 16-element pieces per row
+static MultiShape one_warp_shape(int64_t D, int B, bool nvfp4, int stat)
+{
+    if (D == 2560) return {1, 160};
+    if (D == 512) return {4, 32};
+    if (D == 768 && B == 16) return {2, 48};
+    if (D == 1280 && (nvfp4 || (B == 16 && stat == STAT_MX))) return {2, 80};
+    if (D == 1536 && nvfp4) return {1, 96};
+    return {0, 0};
+}
 
 template <int LPB, int FMT, int STAT>
-static fwd_fn multi_by_rows(int rpw)
+static fwd_fn multi_by_rows(int ch)
 {
-    if constexpr (FMT == 2) return rpw == 1 ? fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT> : fwd_multi_kernel<16, LPB, 5, 2, 80, STAT, FMT>;
-    else return rpw == 1 ? fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT> : nullptr;   // two rows per warp: NVFP4 only
+    if (ch == 160) return fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT>;
+    if (ch == 32) return fwd_multi_kernel<16, LPB, 4, 4, 32, STAT, FMT>;
+    if constexpr (LPB == 1) {
+        if (ch == 48) return fwd_multi_kernel<16, LPB, 3, 2, 48, STAT, FMT>;
+        if constexpr (FMT == 2 || STAT == STAT_MX) {
+            if (ch == 80) return fwd_multi_kernel<16, LPB, 5, 2, 80, STAT, FMT>;
+        }
+        if constexpr (FMT == 2) {
+            if (ch == 96) return fwd_multi_kernel<16, LPB, 3, 1, 96, STAT, FMT>;
+        }
+    }
+    return nullptr;
 }
 template <int FMT, int STAT>
-static fwd_fn pick_multi(int B, int rpw)
+static fwd_fn pick_multi(int B, int ch)
 {
-    if constexpr (FMT == 2) return multi_by_rows<1, 2, STAT>(rpw);
-    else return B == 16 ? multi_by_rows<1, FMT, STAT>(rpw) : B == 32 ? multi_by_rows<2, FMT, STAT>(rpw) : multi_by_rows<4, FMT, STAT>(rpw);
+    if constexpr (FMT == 2) return multi_by_rows<1, 2, STAT>(ch);
+    else return B == 16 ? multi_by_rows<1, FMT, STAT>(ch) : B == 32 ? multi_by_rows<2, FMT, STAT>(ch) : multi_by_rows<4, FMT, STAT>(ch);
 }
 template <int FMT>
-static fwd_fn pick_multi_stat(int B, int stat, int rpw)
+static fwd_fn pick_multi_stat(int B, int stat, int ch)
 {
-    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B, rpw) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B, rpw) : pick_multi<FMT, STAT_NONE>(B, rpw);
+    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B, ch) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B, ch) : pick_multi<FMT, STAT_NONE>(B, ch);
 }
 
 
@@ -484,8 +508,9 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     P.rows_per_cta = rows_per_cta(P.wpr);
     fwd_fn fn = nullptr;
     // (the one-warp kernel has the paper's rounding rule compiled in and takes no gain)
-    if (const int rpw = one_warp_rows(P.D, nvfp4); rpw > 0 && !has_gain && (nvfp4 || mxfp4 || P.round == MXN_ROUND_RCEIL_POW2) && (fine || mxfp4) && stat != STAT_POSTROUND) {
-        fn = nvfp4 ? pick_multi_stat<2>(16, stat, rpw) : mxfp4 ? pick_multi_stat<1>(B, stat, rpw) : pick_multi_stat<0>(B, stat, rpw);
+    if (const MultiShape ms = one_warp_shape(P.D, B, nvfp4, stat); ms.rpw > 0 && !has_gain && (nvfp4 || mxfp4 || P.round == MXN_ROUND_RCEIL_POW2) && (fine || mxfp4) && stat != STAT_POSTROUND) {
+        const int rpw = ms.rpw;
+        fn = nvfp4 ? pick_multi_stat<2>(16, stat, ms.ch) : mxfp4 ? pick_multi_stat<1>(B, stat, ms.ch) : pick_multi_stat<0>(B, stat, ms.ch);
         *fn_out = fn;
         *ctas_out = (P.T + (int64_t)MXN_FWD_WARPS * rpw - 1) / ((int64_t)MXN_FWD_WARPS * rpw);
         *threads_out = MXN_FWD_WARPS * kWarp;

@@ -29,7 +29,9 @@ def rows(T, D, seed, outliers=True):
 SHAPES = [(1, 32), (5, 64), (37, 768), (130, 1024), (9, 2560), (33, 4096), (6, 5120), (5, 8192), (3, 16384),
           (2, 32768), (257, 2048),
           # hidden sizes {3,5,7} * 2^r of the paper's sweep: rows spanning 3, 5, 6 and 7 warps
-          (7, 3072), (5, 6144), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (11, 1280), (9, 1792), (10, 1536), (6, 3584), (133, 1280), (130, 2560)]
+          (7, 3072), (5, 6144), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (11, 1280), (9, 1792), (10, 1536), (6, 3584), (133, 1280), (130, 2560),
+          # several rows per warp (D = 512: four), with a ragged last warp
+          (131, 512), (3, 512)]
 
 
 @pytest.mark.parametrize("T,D", SHAPES)
@@ -63,7 +65,7 @@ def test_rmsnorm_mxfp8_fwd_matches_oracle(binding, oracle, T, D):
 
 @pytest.mark.parametrize("block", [16, 64])
 @pytest.mark.parametrize("T,D", [(3, 64), (19, 1024), (5, 2048), (9, 2560), (130, 2560), (6, 3072), (7, 4096), (4, 8192), (3, 16384),
-                                 (10, 1536), (6, 3584), (11, 1280), (133, 1280),
+                                 (10, 1536), (6, 3584), (11, 1280), (133, 1280), (37, 768), (131, 512),
                                  # with a gain every block size runs as 16-element pieces: rows of 3, 5, 6, 7 and 16 warps
                                  (3, 5120), (5, 6144), (3, 7168), (2, 10240), (2, 12288), (2, 14336), (2, 32768)])
 def test_other_block_sizes(binding, oracle, T, D, block):
@@ -91,7 +93,7 @@ def test_other_rounding_modes(binding, oracle, rnd, T, D):
     gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, round=rnd), f"mxnorm gain round={rnd}")
 
 
-@pytest.mark.parametrize("T,D", [(1, 32), (37, 768), (128, 128), (200, 192), (300, 4096), (129, 2560)])
+@pytest.mark.parametrize("T,D", [(1, 32), (37, 768), (128, 128), (200, 192), (300, 4096), (129, 2560), (131, 512)])
 def test_tiled_scale_layout(binding, oracle, T, D):
     x, _ = rows(T, D, seed=T * 7 + D)
     for kind in ("mx", "cast", "rms"):
@@ -212,7 +214,7 @@ def test_nvfp4_at_the_edge_of_the_stated_domain(binding, oracle):
 
 @pytest.mark.parametrize("T,D", [(1, 16), (5, 48), (37, 768), (130, 1024), (33, 4096), (5, 8192), (3, 16384), (257, 2048),
                                  (7, 3072), (6, 5120), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (11, 1280),
-                                 (9, 2560), (131, 2560), (10, 1536), (6, 3584), (133, 1280)])
+                                 (9, 2560), (131, 2560), (10, 1536), (6, 3584), (133, 1280), (131, 512), (133, 1536)])
 def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
     x, _ = rows(T, D, seed=11 * T + D)
     for p, eps, gs in ((2, 1e-5, 1.0), (1, 0.0, 1.0), (2, 0.0, 8.0)):
@@ -272,7 +274,7 @@ def test_rms_output_is_optional_and_stream_is_honoured(binding, oracle):
 
 @pytest.mark.parametrize("block", [16, 32, 64])
 @pytest.mark.parametrize("T,D", [(1, 64), (37, 768), (130, 1024), (33, 4096), (9, 2560), (5, 8192), (3, 16384), (257, 2048), (133, 1280),
-                                 (7, 3072), (6, 5120), (5, 6144), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (10, 1536), (6, 3584)])
+                                 (7, 3072), (6, 5120), (5, 6144), (4, 7168), (3, 10240), (3, 12288), (3, 14336), (10, 1536), (6, 3584), (131, 512), (7, 512)])
 def test_mxfp4_matches_oracle(binding, oracle, T, D, block):
     """E2M1 codes with E8M0 scales (the paper's cast with the element type set to E2M1)."""
     x, _ = rows(T, D, seed=13 * T + D + block)
