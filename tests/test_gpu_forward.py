@@ -228,6 +228,36 @@ def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
         gu.assert_exact(got, gu.run_ref(oracle, "cast_nvfp4", x, global_scale=gs), f"mx_cast_nvfp4 {T}x{D} g={gs}")
 
 
+@pytest.mark.parametrize("D,blocks", [(512, (16, 32, 64)), (768, (16,)), (1280, (16,))])
+def test_many_short_rows_take_several_rows_per_warp(binding, oracle, D, blocks):
+    """From about twelve thousand rows on, rows of 512, 768 (blocks of 16) and 1280 elements (blocks of 16, MXNorm statistic)
+    run several to a warp; the odd row count leaves the last warp a partial run."""
+    T = 12288 + 5
+    x, _ = rows(T, D, seed=19 + D)
+    for block in blocks:
+        for layout in (0, 1):
+            got = gu.run_fwd(binding, oracle, "mx", x, block=block, eps=1e-5, layout=layout)
+            gu.assert_exact(got, gu.run_ref(oracle, "mx", x, block=block, eps=1e-5), f"mxnorm B={block} layout={layout} {T}x{D}")
+        got = gu.run_fwd(binding, oracle, "mx", x, block=block, p=1)
+        gu.assert_exact(got, gu.run_ref(oracle, "mx", x, block=block, p=1), f"mxnorm p=1 B={block} {T}x{D}")
+        got = gu.run_fwd(binding, oracle, "mx4", x, block=block, eps=1e-5, layout=1)
+        gu.assert_exact(got, gu.run_ref(oracle, "mx4", x, block=block, eps=1e-5), f"mxnorm_mxfp4 B={block} {T}x{D}")
+        if D != 1280:     # the other statistics take this kernel at D = 512 and 768 only
+            got = gu.run_fwd(binding, oracle, "cast", x, block=block)
+            gu.assert_exact(got, gu.run_ref(oracle, "cast", x, block=block), f"mx_cast B={block} {T}x{D}")
+            got = gu.run_fwd(binding, oracle, "cast4", x, block=block)
+            gu.assert_exact(got, gu.run_ref(oracle, "cast4", x, block=block), f"mx_cast_fp4 B={block} {T}x{D}")
+            got = gu.run_fwd(binding, oracle, "rms", x, block=block, eps=1e-5)
+            gu.assert_within_rounding_of_rho(got, gu.run_ref(oracle, "rms", x, block=block, eps=1e-5), block, "rms")
+            got = gu.run_fwd(binding, oracle, "rms4", x, block=block, eps=1e-5)
+            gu.assert_within_rounding_of_rho(got, gu.run_ref(oracle, "rms4", x, block=block, eps=1e-5), block, "rmsnorm_mxfp4", fp4=True)
+    if D != 1280:
+        got = gu.run_fwd(binding, oracle, "nvfp4", x, eps=1e-5, layout=1)
+        gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x, eps=1e-5), f"nvfp4 {T}x{D}")
+        got = gu.run_fwd(binding, oracle, "cast_nvfp4", x, global_scale=0.25)
+        gu.assert_exact(got, gu.run_ref(oracle, "cast_nvfp4", x, global_scale=0.25), f"mx_cast_nvfp4 {T}x{D}")
+
+
 def test_gain_is_applied_after_the_normaliser(binding, oracle):
     """Rows on which (x * rho~) * gamma and (x * gamma) * rho~ round to different E4M3 codes (found by search; the CPU pin of
     the oracle uses the same rows): the kernels must take the first order, for MXNorm and for the conventional path."""
