@@ -85,6 +85,11 @@ def test_random_cases_match_the_oracle_bit_for_bit(binding, oracle, seed):
         gu.assert_exact(got, gu.run_ref(oracle, "mx4", x, block=block, p=p, eps=eps), "mxnorm_mxfp4_fwd " + what)
         got = gu.run_fwd(binding, oracle, "cast4", x, block=block, layout=layout)
         gu.assert_exact(got, gu.run_ref(oracle, "cast4", x, block=block), "mx_cast_fp4 " + what)
+        # gain vector: magnitudes over twenty binades, both signs, some exact zeros
+        g = rng.standard_normal(D) * 2.0 ** rng.uniform(-10, 10, size=D) * (rng.random(D) > 0.02)
+        gain = f32_to_bf16_bits(g)
+        got = gu.run_fwd(binding, oracle, "mx", x, gain, block=block, p=p, eps=eps, round=rnd, layout=layout)
+        gu.assert_exact(got, gu.run_ref(oracle, "mx", x, gain, block=block, p=p, eps=eps, round=rnd), f"mxnorm_fwd with gain round={rnd} " + what)
         if D % 16 == 0:
             got = gu.run_fwd(binding, oracle, "nvfp4", x, p=p, eps=eps, layout=layout)
             gu.assert_exact(got, gu.run_ref(oracle, "nvfp4", x, p=p, eps=eps), "mxnorm_nvfp4_fwd " + what)
