@@ -383,32 +383,37 @@ static fwd_fn pick_e5m2(int wpr, int npass)
 // at 64 registers; [16384, D] and [65536, D]):
 //   D = 2560 (160 pieces, one row per warp: five passes of one warp instead of three warps x one pass or two warps x four
 //     passes): every format, 8-16 % faster;
-//   D = 512 (32 pieces, four rows per warp): every format and statistic, 8-58 % faster at 65536 rows, -8 ... +18 % at 16384;
+//   D = 512 (four rows per warp; 32-element pieces for blocks of 32 and 64 with E8M0 scales, 3-16 % faster than
+//     16-element pieces there): every format and statistic, 8-58 % faster at 65536 rows, -8 ... +18 % at 16384;
 //   D = 768 (48 pieces, two rows per warp): blocks of 16 only (1-19 % faster; blocks of 32 and 64 are level);
 //   D = 1280 (80 pieces, two rows per warp): blocks of 16 with the MXNorm statistic (4-11 % faster; the sum of squares
 //     loses 2-9 % there, blocks of 32 / 64 gain 4 % at 65536 rows and lose 4 % at 16384), and NVFP4 (level);
 //   D = 1536 (96 pieces, one row per warp, three passes): NVFP4 only (6-9 % faster; the E8M0-scaled formats are level).
-// Measured and not kept: two rows of 64 pieces per warp (D = 1024: -9 ... +6 %), 8-element pieces with four lanes per
+// Measured and not kept: two rows per warp at D = 1024 (16-element pieces: -9 ... +6 %; 32-element pieces: -5 ... +3 %), 8-element pieces with four lanes per
 // block (D = 1280: 5.1 -> 3.8 TB/s, D = 1792: 6.1 -> 4.0), and CTA tiles of whole rows packed across warps through shared
 // memory (two CTA-wide barriers per tile: slower than one row per row group at every size but D = 2560).
-struct MultiShape { int rpw, ch; };   // rows per warp, 16-element pieces per row
+struct MultiShape { int rpw, ch, e; };   // rows per warp, pieces per row, elements per piece
 static MultiShape one_warp_shape(int64_t T, int64_t D, int B, bool nvfp4, int stat)
 {
-    if (D == 2560) return {1, 160};
-    if (D == 1280 && nvfp4) return {2, 80};
-    if (D == 1536 && nvfp4) return {1, 96};
+    if (D == 2560) return {1, 160, 16};
+    if (D == 1280 && nvfp4) return {2, 80, 16};
+    if (D == 1536 && nvfp4) return {1, 96, 16};
     // several rows per warp mean as many times fewer CTAs: below about 12 thousand rows the grid no longer fills the
     // SMs (D = 1280, blocks of 16: 9 % slower at 8192 rows, 6-17 % faster from 16384 on)
-    if (T < 12288) return {0, 0};
-    if (D == 512) return {4, 32};
-    if (D == 768 && B == 16) return {2, 48};
-    if (D == 1280 && B == 16 && stat == STAT_MX) return {2, 80};
-    return {0, 0};
+    if (T < 12288) return {0, 0, 0};
+    if (D == 512) return B >= 32 && !nvfp4 ? MultiShape{4, 16, 32} : MultiShape{4, 32, 16};
+    if (D == 768 && B == 16) return {2, 48, 16};
+    if (D == 1280 && B == 16 && stat == STAT_MX) return {2, 80, 16};
+    return {0, 0, 0};
 }
 
 template <int LPB, int FMT, int STAT>
-static fwd_fn multi_by_rows(int ch)
+static fwd_fn multi_by_rows(int ch, int e)
 {
+    if constexpr (LPB >= 2 && FMT != 2) {   // 32-element pieces: a block of 32 is one lane's, a block of 64 two lanes'
+        if (e == 32) return ch == 16 ? fwd_multi_kernel<32, LPB / 2, 2, 4, 16, STAT, FMT> : nullptr;
+    }
+    if (e != 16) return nullptr;
     if (ch == 160) return fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT>;
     if (ch == 32) return fwd_multi_kernel<16, LPB, 4, 4, 32, STAT, FMT>;
     if constexpr (LPB == 1) {
@@ -423,15 +428,15 @@ static fwd_fn multi_by_rows(int ch)
     return nullptr;
 }
 template <int FMT, int STAT>
-static fwd_fn pick_multi(int B, int ch)
+static fwd_fn pick_multi(int B, int ch, int e)
 {
-    if constexpr (FMT == 2) return multi_by_rows<1, 2, STAT>(ch);
-    else return B == 16 ? multi_by_rows<1, FMT, STAT>(ch) : B == 32 ? multi_by_rows<2, FMT, STAT>(ch) : multi_by_rows<4, FMT, STAT>(ch);
+    if constexpr (FMT == 2) return multi_by_rows<1, 2, STAT>(ch, e);
+    else return B == 16 ? multi_by_rows<1, FMT, STAT>(ch, e) : B == 32 ? multi_by_rows<2, FMT, STAT>(ch, e) : multi_by_rows<4, FMT, STAT>(ch, e);
 }
 template <int FMT>
-static fwd_fn pick_multi_stat(int B, int stat, int ch)
+static fwd_fn pick_multi_stat(int B, int stat, int ch, int e)
 {
-    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B, ch) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B, ch) : pick_multi<FMT, STAT_NONE>(B, ch);
+    return stat == STAT_MX ? pick_multi<FMT, STAT_MX>(B, ch, e) : stat == STAT_RMS ? pick_multi<FMT, STAT_RMS>(B, ch, e) : pick_multi<FMT, STAT_NONE>(B, ch, e);
 }
 
 
@@ -514,7 +519,7 @@ static bool select_fwd(FwdParams& P, int B, int stat, bool nvfp4, fwd_fn* fn_out
     // (the one-warp kernel has the paper's rounding rule compiled in and takes no gain)
     if (const MultiShape ms = one_warp_shape(P.T, P.D, B, nvfp4, stat); ms.rpw > 0 && !has_gain && (nvfp4 || mxfp4 || P.round == MXN_ROUND_RCEIL_POW2) && (fine || mxfp4) && stat != STAT_POSTROUND) {
         const int rpw = ms.rpw;
-        fn = nvfp4 ? pick_multi_stat<2>(16, stat, ms.ch) : mxfp4 ? pick_multi_stat<1>(B, stat, ms.ch) : pick_multi_stat<0>(B, stat, ms.ch);
+        fn = nvfp4 ? pick_multi_stat<2>(16, stat, ms.ch, ms.e) : mxfp4 ? pick_multi_stat<1>(B, stat, ms.ch, ms.e) : pick_multi_stat<0>(B, stat, ms.ch, ms.e);
         *fn_out = fn;
         *ctas_out = (P.T + (int64_t)MXN_FWD_WARPS * rpw - 1) / ((int64_t)MXN_FWD_WARPS * rpw);
         *threads_out = MXN_FWD_WARPS * kWarp;
