@@ -385,7 +385,10 @@ static fwd_fn pick_e5m2(int wpr, int npass)
 //     passes): every format, 8-16 % faster;
 //   D = 512 (four rows per warp; 32-element pieces for blocks of 32 and 64 with E8M0 scales, 3-16 % faster than
 //     16-element pieces there): every format and statistic, 8-58 % faster at 65536 rows, -8 ... +18 % at 16384;
-//   D = 768 (48 pieces, two rows per warp): blocks of 16 only (1-19 % faster; blocks of 32 and 64 are level);
+//   D = 256 (eight rows per warp, pieces as for D = 512): every format, 10-127 % faster from 32768 rows on (a row of
+//     256 elements leaves three quarters of a warp's lanes idle in the row-group kernels);
+//   D = 768 (48 pieces, two rows per warp): blocks of 16 only (1-19 % faster; blocks of 32 and 64 are level, also as
+//     32-element pieces);
 //   D = 1280 (80 pieces, two rows per warp): blocks of 16 with the MXNorm statistic (4-11 % faster; the sum of squares
 //     loses 2-9 % there, blocks of 32 / 64 gain 4 % at 65536 rows and lose 4 % at 16384), and NVFP4 (level);
 //   D = 1536 (96 pieces, one row per warp, three passes): NVFP4 only (6-9 % faster; the E8M0-scaled formats are level).
@@ -398,9 +401,11 @@ static MultiShape one_warp_shape(int64_t T, int64_t D, int B, bool nvfp4, int st
     if (D == 2560) return {1, 160, 16};
     if (D == 1280 && nvfp4) return {2, 80, 16};
     if (D == 1536 && nvfp4) return {1, 96, 16};
-    // several rows per warp mean as many times fewer CTAs: below about 12 thousand rows the grid no longer fills the
-    // SMs (D = 1280, blocks of 16: 9 % slower at 8192 rows, 6-17 % faster from 16384 on)
+    // several rows per warp mean as many times fewer CTAs: below about 12 thousand rows (24 thousand for eight rows per
+    // warp) the grid no longer fills the SMs (D = 1280, blocks of 16: 9 % slower at 8192 rows, 6-17 % faster from 16384 on;
+    // D = 256: -10 ... +27 % at 16384 rows, 10-127 % faster from 32768 on)
     if (T < 12288) return {0, 0, 0};
+    if (D == 256 && T >= 24576) return B >= 32 && !nvfp4 ? MultiShape{8, 8, 32} : MultiShape{8, 16, 16};
     if (D == 512) return B >= 32 && !nvfp4 ? MultiShape{4, 16, 32} : MultiShape{4, 32, 16};
     if (D == 768 && B == 16) return {2, 48, 16};
     if (D == 1280 && B == 16 && stat == STAT_MX) return {2, 80, 16};
@@ -411,11 +416,12 @@ template <int LPB, int FMT, int STAT>
 static fwd_fn multi_by_rows(int ch, int e)
 {
     if constexpr (LPB >= 2 && FMT != 2) {   // 32-element pieces: a block of 32 is one lane's, a block of 64 two lanes'
-        if (e == 32) return ch == 16 ? fwd_multi_kernel<32, LPB / 2, 2, 4, 16, STAT, FMT> : nullptr;
+        if (e == 32) return ch == 16 ? fwd_multi_kernel<32, LPB / 2, 2, 4, 16, STAT, FMT> : ch == 8 ? fwd_multi_kernel<32, LPB / 2, 2, 8, 8, STAT, FMT> : nullptr;
     }
     if (e != 16) return nullptr;
     if (ch == 160) return fwd_multi_kernel<16, LPB, 5, 1, 160, STAT, FMT>;
     if (ch == 32) return fwd_multi_kernel<16, LPB, 4, 4, 32, STAT, FMT>;
+    if (ch == 16) return fwd_multi_kernel<16, LPB, 4, 8, 16, STAT, FMT>;
     if constexpr (LPB == 1) {
         if (ch == 48) return fwd_multi_kernel<16, LPB, 3, 2, 48, STAT, FMT>;
         if constexpr (FMT == 2 || STAT == STAT_MX) {

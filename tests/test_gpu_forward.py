@@ -228,11 +228,11 @@ def test_nvfp4_matches_oracle_bit_for_bit(binding, oracle, T, D):
         gu.assert_exact(got, gu.run_ref(oracle, "cast_nvfp4", x, global_scale=gs), f"mx_cast_nvfp4 {T}x{D} g={gs}")
 
 
-@pytest.mark.parametrize("D,blocks", [(512, (16, 32, 64)), (768, (16,)), (1280, (16,))])
-def test_many_short_rows_take_several_rows_per_warp(binding, oracle, D, blocks):
+@pytest.mark.parametrize("D,blocks,T", [(512, (16, 32, 64), 12288 + 5), (768, (16,), 12288 + 5), (1280, (16,), 12288 + 5),
+                                        (256, (16, 32, 64), 24576 + 5)])
+def test_many_short_rows_take_several_rows_per_warp(binding, oracle, D, blocks, T):
     """From about twelve thousand rows on, rows of 512, 768 (blocks of 16) and 1280 elements (blocks of 16, MXNorm statistic)
-    run several to a warp; the odd row count leaves the last warp a partial run."""
-    T = 12288 + 5
+    run several to a warp, from twenty-four thousand on rows of 256 too; the odd row count leaves the last warp a partial run."""
     x, _ = rows(T, D, seed=19 + D)
     for block in blocks:
         for layout in (0, 1):
