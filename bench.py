@@ -119,12 +119,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_launches(fn, n_sets: int, steps: int, warmup: int, stream) -> float:
-    """Average device milliseconds per call of fn(set_index) over `steps` back-to-back launches."""
+GATE_CYCLES = 200_000      # about 0.1 ms of a clock-spin kernel in front of a timed region (see time_launches)
+
+
+def time_launches(fn, n_sets: int, steps: int, warmup: int, stream, gate: bool = True) -> float:
+    """Average device milliseconds per call of fn(set_index) over `steps` back-to-back launches.
+
+    After the synchronize the GPU is idle, and an event recorded then is stamped at once while the first timed launch is
+    still on its way from the host (some 10 us, which a region of 20 launches of 30 us would carry as +1.5 %).  With
+    `gate` a short clock-spin kernel is enqueued first: the host queues the timed launches behind it, and the start event
+    is stamped when the first of them can begin."""
     for i in range(warmup):
         fn(i % n_sets)
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    if gate:
+        with torch.cuda.stream(stream):
+            torch.cuda._sleep(GATE_CYCLES)
     start.record(stream)
     for i in range(steps):
         fn(i % n_sets)
@@ -141,6 +152,7 @@ def time_repeated(fn, n_sets: int, steps: int, warmup: int, stream, repeats: int
 
 
 REST_S = 0.5        # idle time before a secondary kernel is timed (see time_median)
+OTHERS_MIN_STEPS = 100   # launches per timed region of a secondary kernel, at least
 
 
 def time_median(fn, n_sets: int, steps: int, warmup: int, stream, repeats: int = 3) -> float:
@@ -396,8 +408,11 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(T, D),
                    "l2": f"inputs/outputs rotate over {SETS} buffer sets ({SETS * nbytes / 1e6:.0f} MB > 126 MB L2)",
-                   "timing": f"{REPEATS} timed regions of {args.steps} launches each after {args.warmup} warm-up launches; ms_per_step "
-                             "is the median region, ms_per_step_spread its minimum and maximum; the other kernels: median of 3 regions, each kernel "
+                   "timing": f"{REPEATS} timed regions of {args.steps} launches each after {args.warmup} warm-up launches, every region bracketed by a "
+                             "device synchronize and started behind a 0.1 ms clock-spin kernel so that the start event is not stamped "
+                             "while the first launch is still on its way from the host; ms_per_step "
+                             "is the median region, ms_per_step_spread its minimum and maximum; the other kernels: median of 3 regions of "
+                             f"max(steps, {OTHERS_MIN_STEPS}) launches (half as many for the backward), each kernel "
                              f"after {REST_S} s of idle (burst figures, like the measured copy peak; seconds into an uninterrupted load "
                              "the instruction-heavier kernels run up to 8 % slower on this pool)",
                    "launch": "back-to-back launches in one stream, as the library issues them: programmatic stream "
@@ -421,11 +436,16 @@ def main():
     if not args.skip_others:
         # ---- the rest of the path, each timed the same way (context for the headline) ----
         others = {}
-        ms_rms = time_median(rms, SETS, args.steps, args.warmup, stream)
-        ms_cast = time_median(cast, SETS, args.steps, args.warmup, stream)
+        # regions of at least OTHERS_MIN_STEPS launches whatever --steps says: a region of 10-20 launches carries the ramp
+        # of its first and the tail of its last launch as 1-2 % (the headline keeps exactly --steps launches per region)
+        osteps = max(args.steps, OTHERS_MIN_STEPS)
+        ms_rms = time_median(rms, SETS, osteps, args.warmup, stream)
+        ms_cast = time_median(cast, SETS, osteps, args.warmup, stream)
+        ms_fwd_same = time_median(fwd, SETS, osteps, args.warmup, stream)      # the headline kernel timed the same way, for the ratio
         others["rmsnorm_mxfp8_fwd"] = {"ms": ms_rms, "gbs": algorithmic_bytes("rms", T, D) / ms_rms / 1e6}
         others["mx_cast"] = {"ms": ms_cast, "gbs": algorithmic_bytes("cast", T, D) / ms_cast / 1e6}
-        result["speedup_vs_rmsnorm_mxfp8_fwd"] = ms_rms / ms
+        others["mxnorm_fwd"] = {"ms": ms_fwd_same, "gbs": nbytes / ms_fwd_same / 1e6}
+        result["speedup_vs_rmsnorm_mxfp8_fwd"] = ms_rms / ms_fwd_same
         def time_secondary_kernels():
             # NVFP4
             o4 = [mx.alloc_outputs(T, D, 16, mx.SCALES_ROWMAJOR, nvfp4=True) for _ in range(SETS)]
@@ -442,8 +462,8 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            ms4 = time_median(nvfp4, SETS, args.steps, args.warmup, stream)
-            ms4r = time_median(rms_nvfp4, SETS, args.steps, args.warmup, stream)
+            ms4 = time_median(nvfp4, SETS, osteps, args.warmup, stream)
+            ms4r = time_median(rms_nvfp4, SETS, osteps, args.warmup, stream)
             others["mxnorm_nvfp4_fwd"] = {"ms": ms4, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4 / 1e6}
             others["rmsnorm_nvfp4_fwd"] = {"ms": ms4r, "gbs": algorithmic_bytes("nvfp4", T, D) / ms4r / 1e6}
             result["nvfp4_speedup_vs_rmsnorm_nvfp4_fwd"] = ms4r / ms4
@@ -457,7 +477,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msm4 = time_median(mxfp4, SETS, args.steps, args.warmup, stream)
+            msm4 = time_median(mxfp4, SETS, osteps, args.warmup, stream)
             others["mxnorm_mxfp4_fwd"] = {"ms": msm4, "gbs": (T * D * 2 + T * D // 2 + T * (D // 32) + 4 * T) / msm4 / 1e6}
             del m4
             if T % 32 == 0:
@@ -470,7 +490,7 @@ def main():
                     if st != 0:
                         raise RuntimeError(mx.status_string(st))
 
-                mst = time_median(transposed, SETS, args.steps, args.warmup, stream)
+                mst = time_median(transposed, SETS, osteps, args.warmup, stream)
                 others["mx_cast_transposed"] = {"ms": mst, "gbs": (T * D * 3 + T * D // 32 + 4 * T) / mst / 1e6}
 
                 def transposed_plain(i):   # no normaliser: the column-wise cast of the upstream gradient
@@ -478,7 +498,7 @@ def main():
                     if st != 0:
                         raise RuntimeError(mx.status_string(st))
 
-                mstp = time_median(transposed_plain, SETS, args.steps, args.warmup, stream)
+                mstp = time_median(transposed_plain, SETS, osteps, args.warmup, stream)
                 others["mx_cast_transposed_no_normaliser"] = {"ms": mstp, "gbs": (T * D * 3 + T * D // 32) / mstp / 1e6}
                 del ct, stt
             # the ablation with power-of-two-rounded block maxima, and the residual add fused in front
@@ -488,7 +508,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            mspr = time_median(postround, SETS, args.steps, args.warmup, stream)
+            mspr = time_median(postround, SETS, osteps, args.warmup, stream)
             others["mxnorm_postround_fwd"] = {"ms": mspr, "gbs": algorithmic_bytes("mx", T, D) / mspr / 1e6}
             # the same two kernels with a gain vector (the extension of Algorithm 2; Algorithm 1 as commonly deployed)
             gain_vec = (1.0 + 0.1 * torch.randn(D, generator=torch.Generator().manual_seed(2))).to(torch.bfloat16).cuda()   # made on the host: no torch kernel
@@ -505,9 +525,9 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msg = time_median(fwd_gain, SETS, args.steps, args.warmup, stream)
+            msg = time_median(fwd_gain, SETS, osteps, args.warmup, stream)
             others["mxnorm_fwd_with_gain"] = {"ms": msg, "gbs": (algorithmic_bytes("mx", T, D) + 2 * D) / msg / 1e6}
-            msg = time_median(rms_gain, SETS, args.steps, args.warmup, stream)
+            msg = time_median(rms_gain, SETS, osteps, args.warmup, stream)
             others["rmsnorm_mxfp8_fwd_with_gain"] = {"ms": msg, "gbs": (algorithmic_bytes("rms", T, D) + 2 * D) / msg / 1e6}
             hs = [torch.empty_like(xs[0]) for _ in range(SETS)]
 
@@ -518,7 +538,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msadd = time_median(add_fwd, SETS, args.steps, args.warmup, stream)
+            msadd = time_median(add_fwd, SETS, osteps, args.warmup, stream)
             others["mxnorm_add_fwd"] = {"ms": msadd, "gbs": (algorithmic_bytes("mx", T, D) + 4 * T * D) / msadd / 1e6}
             del hs
             # backward (C5 tensors: seed 1, gradient ~ N(0, 1e-2), gain)
@@ -541,7 +561,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msb = time_median(bwd, nb, max(10, args.steps // 2), args.warmup, stream)
+            msb = time_median(bwd, nb, max(osteps // 2, 10), args.warmup, stream)
             others["mxnorm_bwd"] = {"ms": msb, "gbs": algorithmic_bytes("bwd", T, D) / msb / 1e6}
 
             def bwd_dx_only(i):   # the method's own configuration: no gain (folded into the next weight), hence no gain gradient
@@ -549,7 +569,7 @@ def main():
                 if st != 0:
                     raise RuntimeError(mx.status_string(st))
 
-            msbx = time_median(bwd_dx_only, nb, max(10, args.steps // 2), args.warmup, stream)
+            msbx = time_median(bwd_dx_only, nb, max(osteps // 2, 10), args.warmup, stream)
             others["mxnorm_bwd_dx_only"] = {"ms": msbx, "gbs": (3 * T * D * 2 + 4 * T) / msbx / 1e6}
             del xb, gb, dxb
 
@@ -577,7 +597,7 @@ def main():
             mx.mxnorm_fwd_host(xh, ch, shh, rh, wsh, eps=EPS, layout=layout, stream=stream)
 
         e2e_steps = max(3, min(args.steps, 20))
-        ms_e2e = time_launches(e2e_step, 1, e2e_steps, 3, stream)
+        ms_e2e = time_launches(e2e_step, 1, e2e_steps, 3, stream, gate=False)   # end to end: the host's latency belongs to it
         ms_e2e = sharding.max_over_ranks(ms_e2e, device="cuda")
         result["e2e"] = {"value": nbytes * world / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms_e2e,
                          "steps": e2e_steps, "h2d_bytes_per_step": T * D * 2,
