@@ -327,7 +327,7 @@ struct BwdPlan { int threads, V, stages, stage_bytes, ctas_per_sm; size_t smem; 
 //   variant (20 or 24 warps per SM); with the gain gradient at most 8 CTAs, because every CTA adds a row of partial sums.
 //   D = 3072: 192 threads x 3 CTAs (49.7 / 44.3 us; 4 CTAs: 64.7 / 45.8).  D = 4096: 256 x 2 (65.2 / 59.2; 3 CTAs: 82.4 / 62.4).
 //   Wider rows: 3 or 4 vectors per thread, 2 CTAs per SM; beyond 8192 elements 512 threads, 1 CTA.
-static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false)
+static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false, int64_t T = 0)
 {
     if (D <= 0 || D % 8 != 0 || D > 16384) return false;
     const int64_t nvec = D / 8;
@@ -349,6 +349,28 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false)
         n = (int)(((nvec + v - 1) / v + 31) / 32 * 32);          // no more threads than v vectors each need (D = 3072: 192, not 256)
         ctas = n > MXN_BWD_THREADS ? 1 : (v == 2 && n <= 192) ? 3 : MXN_BWD_CTAS;
     }
+    // Ring depth and CTAs per SM by row length and row count.  The defaults above were timed at 16384 rows; timing every
+    // hidden size of the paper's grid at 16384, 32768 and 65536 rows with 2, 3 or the default number of stages and with fewer
+    // CTAs per SM showed that long launches and long rows want fewer copies in flight (same DRAM bytes, measured; the DRAM
+    // is busier: 82 % against 77 % of its cycles at [65536, 5120]).  What the rules below buy, default -> rule:
+    //   rows wider than 8192 elements (512 threads): two stages, dX alone 4-10 % faster at 10240 ... 14336, level elsewhere;
+    //   four vectors per thread in 256 threads (D = 7168, 8192) without the gain gradient: one CTA per SM, 3-13 % faster;
+    //   three vectors per thread (D = 5120, 6144): two stages, with the gain gradient always (1-14 % faster), else from
+    //     32768 rows on (5-7 %);
+    //   D = 3072 (two vectors in 192 threads) from 32768 rows on: two stages, 2-10 % faster;
+    //   D <= 1792 with the gain gradient: three stages, 2-11 % faster;
+    //   1536 <= D <= 2048 from 32768 rows on: a third fewer CTAs per SM with deeper rings, 3-20 % faster.
+    // Over the 102 cells the geometric mean is 3 % faster, the worst cell 1.8 % slower (D = 10240, dX alone, 16384 rows).
+    int forced_stages = 0;
+    const bool many_rows = T >= 32768;
+    if (n > MXN_BWD_THREADS) forced_stages = 2;
+    else if (v == 4 && !dgain) ctas = 1;
+    else if (v == 3 && (dgain || many_rows)) forced_stages = 2;
+    else if (v == 2 && n == 192 && nvec > 256 && many_rows) forced_stages = 2;
+    else if (nvec <= 256) {
+        if (dgain && D <= 1792) forced_stages = 3;
+        else if (many_rows && D >= 1536) ctas = ctas >= 8 ? 5 : ctas >= 5 ? 4 : ctas;
+    }
     pl->threads = n;
     pl->V = v;                                                   // 1..4, each instantiated
     pl->ctas_per_sm = ctas;
@@ -356,6 +378,7 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false)
     const int budget = 200 * 1024 / pl->ctas_per_sm;            // shared memory per CTA
     int st = budget / pl->stage_bytes;
     pl->stages = st < 2 ? 2 : (st > kBwdMaxStages ? kBwdMaxStages : st);
+    if (forced_stages != 0 && forced_stages < pl->stages) pl->stages = forced_stages;
     pl->smem = (size_t)pl->stages * pl->stage_bytes;
     if (pl->V == 4 && gain && dgain) {   // room behind the ring for the gain of the variant that parks it there
         const size_t gain_bytes = (size_t)(D * 2 + 127) / 128 * 128;
@@ -374,7 +397,9 @@ bool bwd_shape_supported(int64_t D)
 int bwd_parts(int64_t T, int64_t D)
 {
     BwdPlan pl;
-    if (!plan_bwd(D, true, &pl)) return 0;      // the plan with the gain gradient: the one that needs the workspace
+    // the plan with the gain gradient (the one that needs the workspace) for few rows: it has the most CTAs per SM, so
+    // a workspace sized for T rows also serves every call with fewer rows
+    if (!plan_bwd(D, true, &pl)) return 0;
     const int64_t cap = (int64_t)kSMs * pl.ctas_per_sm;
     return (int)(T < cap ? (T < 1 ? 1 : T) : cap);
 }
@@ -394,7 +419,7 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
 {
     const bool gain = P.gain != nullptr, dgain = P.dgain != nullptr;
     BwdPlan pl;
-    if (!plan_bwd(P.D, dgain, &pl, gain)) return cudaErrorInvalidValue;
+    if (!plan_bwd(P.D, dgain, &pl, gain, P.T)) return cudaErrorInvalidValue;
     P.stages = pl.stages;
     P.stage_bytes = pl.stage_bytes;
     {   // the grid of this variant (with the gain gradient it equals bwd_parts(T, D), which sized the workspace)
@@ -448,17 +473,23 @@ int64_t selftest_bwd_plans(int64_t max_D, int64_t* first_D, int* first_case)
         if (!bwd_shape_supported(D)) continue;
         for (int c = 0; c < 4; ++c) {
             const bool gain = (c & 2) != 0, dgain = (c & 1) != 0;
-            BwdPlan pl;
-            bool ok = plan_bwd(D, dgain, &pl, gain);
-            if (ok) {
-                const size_t ring = (size_t)pl.stages * pl.stage_bytes;
-                const size_t parked = pl.V == 4 && gain && dgain ? (size_t)(D * 2 + 127) / 128 * 128 : 0;
-                ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V == 4))
-                  && pl.threads % 32 == 0 && (int64_t)pl.threads * pl.V >= D / 8 && pl.stages >= 2 && pl.stages <= kBwdMaxStages
-                  && pl.stage_bytes >= 4 * D && pl.smem == ring + parked
-                  && pl.smem <= 227 * 1024                                             // one CTA's limit
-                  && (pl.smem + 2048) * pl.ctas_per_sm <= 228 * 1024                   // the SM's, with static and reserved bytes
-                  && pl.threads * pl.ctas_per_sm <= 2048;
+            bool ok = true;
+            for (int big = 0; big < 2 && ok; ++big) {   // the plan depends on the number of rows
+                const int64_t T = big ? (int64_t)1 << 20 : 1;
+                BwdPlan pl;
+                ok = plan_bwd(D, dgain, &pl, gain, T);
+                if (ok) {
+                    const size_t ring = (size_t)pl.stages * pl.stage_bytes;
+                    const size_t parked = pl.V == 4 && gain && dgain ? (size_t)(D * 2 + 127) / 128 * 128 : 0;
+                    BwdPlan ws;
+                    ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V == 4))
+                      && pl.threads % 32 == 0 && (int64_t)pl.threads * pl.V >= D / 8 && pl.stages >= 2 && pl.stages <= kBwdMaxStages
+                      && pl.stage_bytes >= 4 * D && pl.smem == ring + parked
+                      && pl.smem <= 227 * 1024                                             // one CTA's limit
+                      && (pl.smem + 2048) * pl.ctas_per_sm <= 228 * 1024                   // the SM's, with static and reserved bytes
+                      && pl.threads * pl.ctas_per_sm <= 2048
+                      && plan_bwd(D, true, &ws) && (!dgain || pl.ctas_per_sm <= ws.ctas_per_sm);   // the workspace is sized by the few-rows plan
+                }
             }
             if (!ok && bad++ == 0) {
                 *first_D = D;

@@ -73,6 +73,24 @@ def check(binding, oracle, T, D, seed, with_gain=True):
     return dx, dg
 
 
+@pytest.mark.parametrize("D", [1536, 2048, 3072])
+def test_backward_with_many_rows(binding, oracle, D):
+    """From 32768 rows on the launcher takes fewer CTAs per SM or a shallower ring for some row lengths: every row of dX
+    and the gain gradient against the oracle, with and without the gain gradient (the two use different launch plans)."""
+    T = 32768 + 3
+    w = wl.Workload("t", T, D, seed=40 + D, outlier_frac=0.002, has_gain=True, has_grad=True)
+    inp = wl.make_inputs(w)
+    x, g, gain = wl.bits(inp["x"]), wl.bits(inp["grad"]), wl.bits(inp["gain"])
+    _, _, rms = oracle.mxnorm_ref(x, eps=1e-5)
+    want_dx, want_dg = oracle.mxnorm_bwd_ref(x, g, gain, rms)
+    row_scale = np.abs(want_dx).max(-1, keepdims=True)
+    dx, _, dg = run_bwd(binding, x, g, gain, rms, fp32_out=True)
+    assert np.max(np.abs(dx - want_dx) / row_scale) < 1e-5
+    assert np.all(np.abs(dg - want_dg) <= 1e-3 * np.abs(want_dg).max())
+    dx2, _, none = run_bwd(binding, x, g, gain, rms, fp32_out=True, want_dgain=False)
+    assert none is None and np.array_equal(dx2, dx)
+
+
 @pytest.mark.parametrize("T,D", [(1, 8), (3, 64), (37, 768), (130, 1024), (65, 2048), (33, 4096), (7, 2056),
                                  (5, 8192), (4, 16384), (1000, 512), (900, 1024), (700, 2048), (9, 5120), (300, 5120), (7, 6144), (300, 8192), (500, 3072), (300, 7168), (450, 1536), (150, 10240), (150, 12288), (150, 14336), (150, 16384)])
 def test_backward_matches_oracle(binding, oracle, T, D):
