@@ -256,7 +256,8 @@ mxn_status mx_cast_transposed_e5m2(const void* x_bf16, int64_t T, int64_t D,
  *   dx = 0 and adds nothing to dgain.
  *   Row sums in binary32; the column sum is a deterministic two-stage reduction through
  *   `workspace` (device memory, >= mxnorm_bwd_workspace_bytes(T, D) bytes, 16-byte aligned;
- *   contents on entry irrelevant, clobbered on exit; may be NULL when dgain is NULL). */
+ *   contents on entry irrelevant, clobbered on exit; may be NULL when dgain is NULL).  The size does not
+ *   decrease with T: a workspace sized for T rows also serves every call with fewer rows of the same D. */
 mxn_status mxnorm_bwd(const void* x_bf16, const void* grad_out_bf16, const void* gain_bf16_or_null,
                       const float* rms, int64_t T, int64_t D,
                       void* dx, int dx_is_fp32, float* dgain_f32_or_null,
