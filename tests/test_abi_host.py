@@ -92,6 +92,13 @@ def test_every_accepted_shape_has_a_kernel(binding):
     assert binding.lib.mxn_selftest_dispatch(4096, None, None, None) == 1
 
 
+def test_backward_workspace_size_does_not_decrease_with_rows(binding):
+    # the launch plan depends on the row count; the workspace a caller sized for T rows must serve fewer rows too
+    for D in (1024, 1536, 2048, 3072, 4096, 5120, 8192, 16384):
+        sizes = [binding.mxnorm_bwd_workspace_bytes(T, D) for T in (1, 7, 300, 2000, 16384, 32768, 65536, 1 << 20)]
+        assert all(a <= b for a, b in zip(sizes, sizes[1:])) and sizes[0] > 0, (D, sizes)
+
+
 def test_binding_module_has_no_fallback():
     src = open(os.path.join(ROOT, "paper_2603_13180_b200", "binding.py")).read()
     assert "oracle" not in src.replace("CPU oracle", "")
