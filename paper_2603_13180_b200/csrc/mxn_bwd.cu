@@ -358,6 +358,7 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false, int6
     //   three vectors per thread (D = 5120, 6144): two stages, with the gain gradient always (1-14 % faster), else from
     //     32768 rows on (5-7 %);
     //   D = 3072 (two vectors in 192 threads) from 32768 rows on: two stages, 2-10 % faster;
+    //   D = 3584, 4096 (two vectors in 224 / 256 threads) with the gain gradient: three stages, 0-3 % faster;
     //   D <= 1792 with the gain gradient: three stages, 2-11 % faster;
     //   1536 <= D <= 2048 from 32768 rows on: a third fewer CTAs per SM with deeper rings, 3-20 % faster.
     // Over the 102 cells the geometric mean is 3 % faster, the worst cell 1.8 % slower (D = 10240, dX alone, 16384 rows).
@@ -367,6 +368,7 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false, int6
     else if (v == 4 && !dgain) ctas = 1;
     else if (v == 3 && (dgain || many_rows)) forced_stages = 2;
     else if (v == 2 && n == 192 && nvec > 256 && many_rows) forced_stages = 2;
+    else if (v == 2 && n > 192 && dgain) forced_stages = 3;
     else if (nvec <= 256) {
         if (dgain && D <= 1792) forced_stages = 3;
         else if (many_rows && D >= 1536) ctas = ctas >= 8 ? 5 : ctas >= 5 ? 4 : ctas;
