@@ -342,9 +342,9 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false, int6
     } else {
         n = MXN_BWD_THREADS;
         v = (int)((nvec + n - 1) / n);
-        if (v > 4) {   // wide rows: up to 512 threads; that kernel exists with four vectors per thread only
+        if (v > 4) {   // wide rows: up to 512 threads, three or four vectors per thread
             if (nvec > 4 * 512) return false;
-            v = 4;
+            v = nvec > 3 * 512 ? 4 : 3;
         }
         n = (int)(((nvec + v - 1) / v + 31) / 32 * 32);          // no more threads than v vectors each need (D = 3072: 192, not 256)
         ctas = n > MXN_BWD_THREADS ? 1 : (v == 2 && n <= 192) ? 3 : MXN_BWD_CTAS;
@@ -430,9 +430,9 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     }
     // the kernel template below must be the one the plan sized shared memory for (the four-vector variant with gain and
     // gain gradient keeps the gain behind the ring): a mismatch is refused here instead of reaching the device
-    if ((pl.threads > MXN_BWD_THREADS ? 4 : pl.V) != pl.V || pl.threads * pl.V < P.D / 8) return cudaErrorInvalidValue;
+    if ((pl.threads > MXN_BWD_THREADS && pl.V != 3 && pl.V != 4) || pl.threads * pl.V < P.D / 8) return cudaErrorInvalidValue;
     bwd_fn fn;
-    if (pl.threads > MXN_BWD_THREADS) fn = pick_bwd<4, 512>(gain, dgain);
+    if (pl.threads > MXN_BWD_THREADS) fn = pl.V == 3 ? pick_bwd<3, 512>(gain, dgain) : pick_bwd<4, 512>(gain, dgain);
     else if (pl.V == 1) fn = pick_bwd<1, MXN_BWD_THREADS>(gain, dgain);
     else if (pl.V == 2) fn = pl.threads <= 192 ? pick_bwd<2, 192>(gain, dgain) : pick_bwd<2, MXN_BWD_THREADS>(gain, dgain);   // 192: registers for 3+ CTAs per SM
     else if (pl.V == 3) fn = pick_bwd<3, MXN_BWD_THREADS>(gain, dgain);
@@ -484,7 +484,7 @@ int64_t selftest_bwd_plans(int64_t max_D, int64_t* first_D, int* first_case)
                     const size_t ring = (size_t)pl.stages * pl.stage_bytes;
                     const size_t parked = pl.V == 4 && gain && dgain ? (size_t)(D * 2 + 127) / 128 * 128 : 0;
                     BwdPlan ws;
-                    ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V == 4))
+                    ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V >= 3))
                       && pl.threads % 32 == 0 && (int64_t)pl.threads * pl.V >= D / 8 && pl.stages >= 2 && pl.stages <= kBwdMaxStages
                       && pl.stage_bytes >= 4 * D && pl.smem == ring + parked
                       && pl.smem <= 227 * 1024                                             // one CTA's limit
