@@ -346,6 +346,12 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false, int6
             if (nvec > 4 * 512) return false;
             v = nvec > 3 * 512 ? 4 : 3;
         }
+        // D = 8192 with the gain gradient: 512 threads x two vectors in one CTA per SM instead of 256 x four in two (the
+        // four-vector variant with gain and gain gradient recomputes and parks the gain): 133.6 -> 127 us at 16384 rows,
+        // 536 -> 480 us at 65536; narrower rows lose with it (D = 7168: 113 -> 121 us)
+        // (taken without the gain gradient too, where it is level - 118.7 / 119.5 us - so that dX does not depend on
+        // whether the gain gradient is asked for: the order of the row sum follows the thread layout)
+        if (nvec > 960 && nvec <= 1024) v = 2;
         n = (int)(((nvec + v - 1) / v + 31) / 32 * 32);          // no more threads than v vectors each need (D = 3072: 192, not 256)
         ctas = n > MXN_BWD_THREADS ? 1 : (v == 2 && n <= 192) ? 3 : MXN_BWD_CTAS;
     }
@@ -364,7 +370,8 @@ static bool plan_bwd(int64_t D, bool dgain, BwdPlan* pl, bool gain = false, int6
     // Over the 102 cells the geometric mean is 3 % faster, the worst cell 1.8 % slower (D = 10240, dX alone, 16384 rows).
     int forced_stages = 0;
     const bool many_rows = T >= 32768;
-    if (n > MXN_BWD_THREADS) forced_stages = 2;
+    if (n > MXN_BWD_THREADS && v >= 3) forced_stages = 2;
+    else if (n > MXN_BWD_THREADS) forced_stages = 0;
     else if (v == 4 && !dgain) ctas = 1;
     else if (v == 3 && (dgain || many_rows)) forced_stages = 2;
     else if (v == 2 && n == 192 && nvec > 256 && many_rows) forced_stages = 2;
@@ -431,9 +438,9 @@ cudaError_t launch_bwd(BwdParams P, cudaStream_t stream)
     }
     // the kernel template below must be the one the plan sized shared memory for (the four-vector variant with gain and
     // gain gradient keeps the gain behind the ring): a mismatch is refused here instead of reaching the device
-    if ((pl.threads > MXN_BWD_THREADS && pl.V != 3 && pl.V != 4) || pl.threads * pl.V < P.D / 8) return cudaErrorInvalidValue;
+    if ((pl.threads > MXN_BWD_THREADS && (pl.V < 2 || pl.V > 4)) || pl.threads * pl.V < P.D / 8) return cudaErrorInvalidValue;
     bwd_fn fn;
-    if (pl.threads > MXN_BWD_THREADS) fn = pl.V == 3 ? pick_bwd<3, 512>(gain, dgain) : pick_bwd<4, 512>(gain, dgain);
+    if (pl.threads > MXN_BWD_THREADS) fn = pl.V == 2 ? pick_bwd<2, 512>(gain, dgain) : pl.V == 3 ? pick_bwd<3, 512>(gain, dgain) : pick_bwd<4, 512>(gain, dgain);
     else if (pl.V == 1) fn = pick_bwd<1, MXN_BWD_THREADS>(gain, dgain);
     else if (pl.V == 2) fn = pl.threads <= 192 ? pick_bwd<2, 192>(gain, dgain) : pick_bwd<2, MXN_BWD_THREADS>(gain, dgain);   // 192: registers for 3+ CTAs per SM
     else if (pl.V == 3) fn = pick_bwd<3, MXN_BWD_THREADS>(gain, dgain);
@@ -485,7 +492,7 @@ int64_t selftest_bwd_plans(int64_t max_D, int64_t* first_D, int* first_case)
                     const size_t ring = (size_t)pl.stages * pl.stage_bytes;
                     const size_t parked = pl.V == 4 && gain && dgain ? (size_t)(D * 2 + 127) / 128 * 128 : 0;
                     BwdPlan ws;
-                    ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V >= 3))
+                    ok = pl.V >= 1 && pl.V <= 4 && (pl.threads <= MXN_BWD_THREADS || (pl.threads <= 512 && pl.V >= 2))
                       && pl.threads % 32 == 0 && (int64_t)pl.threads * pl.V >= D / 8 && pl.stages >= 2 && pl.stages <= kBwdMaxStages
                       && pl.stage_bytes >= 4 * D && pl.smem == ring + parked
                       && pl.smem <= 227 * 1024                                             // one CTA's limit
